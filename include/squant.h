@@ -1,0 +1,142 @@
+/*
+ * squant.h - C ABI of the B200 (sm_100a) SQuant weight quantizer.
+ *
+ * The library turns the fp32 weights of convolution / fully connected layers into low-bit
+ * integer codes with the progressive solver of the SQuant paper (arXiv 2202.07471,
+ * Algorithm 1 "Progressive SQuant Algorithm"):
+ *
+ *   scale     per output channel, symmetric:  s_m = max|W[m]| / qmax,  qmax = 2^(bits-1) - 1
+ *             (the paper takes s as an input of Algorithm 1 and sets the range per output
+ *             channel, Sec. 4; a channel with max|W| < 2^-100 gets s_m = 1 and all-zero codes)
+ *   SQuant-E  Eq. 9 / Algorithm 1 "Scale and SQuant-E": x = w / s_m in IEEE fp32, round to
+ *             nearest (ties to even); perturbation p = code - x, held as the integer
+ *             nearbyint(p * 2^30) from here on, so that all sums are exact
+ *   SQuant-K  Eq. 10 / Algorithm 2 (SQuantFlip) on each kernel W[m][n][:]: with e the sum of the
+ *             kernel's perturbations, flip the k = round(|e|) elements that have the sign of
+ *             e and the largest |p| by one step, which brings |e| to at most 0.5
+ *   update    Algorithm 3 (UpdatePerturbation): each kernel keeps ONE candidate element for
+ *             SQuant-C (Over SQuant: the last flipped element, to be flipped back;
+ *             Under SQuant: the first un-flipped one)
+ *   SQuant-C  Eq. 11 / Algorithm 2 on each output channel: with e_c the sum of ALL perturbations
+ *             of the channel, flip the candidates of the k_c = round(|e_c|) kernels whose
+ *             candidate has the sign of e_c and the largest |p|, one element per kernel
+ *
+ * Tie rules: round(|e|) at exactly one half takes the smaller count; equal |p| go to the lower
+ * flat index (offset n*K + i inside the output channel).  Results are deterministic and do
+ * not depend on launch geometry.
+ *
+ * Layout: weights and codes are row-major [cout][cin][kh][kw] (a fully connected layer is
+ * kh = kw = 1; a depthwise convolution has cin = 1).  One "kernel" is the kh*kw weights
+ * W[m][n][:], one "output channel" the cin*kh*kw weights W[m][:][:].
+ *
+ * Threading: calls may come from several host threads; the library serialises its own
+ * bookkeeping.  All work is asynchronous on the given CUDA stream unless stated otherwise.
+ */
+#ifndef SQUANT_H_
+#define SQUANT_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* stages to run (bit mask); SQUANT_MODE_E is mandatory */
+#define SQUANT_MODE_E 1u
+#define SQUANT_MODE_K 2u
+#define SQUANT_MODE_C 4u
+#define SQUANT_MODE_EKC (SQUANT_MODE_E | SQUANT_MODE_K | SQUANT_MODE_C)
+
+/* flags */
+#define SQUANT_FLAG_NARROW_RANGE 1u /* codes in [-qmax, qmax] (default); without it the lower
+                                       bound is -qmax-1, which the absmax scale never reaches */
+
+/* error codes (0 = success) */
+#define SQUANT_OK 0
+#define SQUANT_ERR_NULL (-1)        /* a required pointer is NULL */
+#define SQUANT_ERR_SHAPE (-2)       /* a dimension is <= 0 or the element count overflows */
+#define SQUANT_ERR_BITS (-3)        /* bits outside 2..8 */
+#define SQUANT_ERR_MODE (-4)        /* mode mask without SQUANT_MODE_E, unknown bits, or a
+                                       combination that is not built (E|C on kernels > 1x1) */
+#define SQUANT_ERR_ALIGN (-5)       /* weights / scales / error pointers not 4-byte aligned */
+#define SQUANT_ERR_TOO_WIDE (-6)    /* one output channel does not fit the on-chip path */
+#define SQUANT_ERR_CUDA (-7)        /* a CUDA runtime call failed; see squant_last_cuda_error() */
+#define SQUANT_ERR_NOMEM (-8)       /* host or device allocation failed */
+
+typedef struct squant_options {
+    int32_t bits;   /* 2..8; qmax = 2^(bits-1) - 1 */
+    uint32_t mode;  /* SQUANT_MODE_* mask; 0 means SQUANT_MODE_EKC */
+    uint32_t flags; /* SQUANT_FLAG_* */
+} squant_options;
+
+/*
+ * One layer.  For squant_quantize_layer / squant_quantize_model every pointer is a DEVICE
+ * pointer; for squant_quantize_model_host every pointer is a HOST pointer.  The caller owns
+ * all buffers; the library never frees or retains them beyond the call's work on the stream.
+ */
+typedef struct squant_layer {
+    const float *w;      /* in : [cout][cin][kh][kw] fp32, finite values, 4-byte aligned
+                                 (16-byte alignment of every channel enables the fast loads) */
+    int32_t cout, cin, kh, kw;
+    int8_t *codes;       /* out: [cout][cin][kh][kw] int8 */
+    float *scales;       /* out: [cout] */
+    float *kernel_err;   /* out, may be NULL: [cout][cin] final signed sum of a kernel's
+                                 perturbations, (float)(integer sum) * 2^-30 */
+    float *channel_err;  /* out, may be NULL: [cout] final signed sum of a channel's
+                                 perturbations */
+} squant_layer;
+
+/*
+ * Algorithm 1 on one layer (DEVICE pointers).  Same as squant_quantize_model with one layer.
+ */
+int squant_quantize_layer(const squant_layer *layer, const squant_options *opt, void *cuda_stream);
+
+/*
+ * Algorithm 1 on every layer of a model in ONE grouped kernel launch (the paper sums
+ * per-layer times and notes that layers could be quantized in parallel, Sec. 4.2).
+ *
+ *   layers, n_layers  host array of descriptors holding DEVICE pointers; n_layers >= 0
+ *   opt               bits / mode / flags shared by all layers; NULL means 4 bit, E|K|C, narrow
+ *   cuda_stream       a cudaStream_t (NULL = default stream)
+ *
+ * The first call with a given (device, descriptors, options) combination builds a launch plan:
+ * it allocates a small device table and synchronises the stream once.  Later calls with the
+ * same combination only enqueue the kernel.  Outputs are valid when the stream reaches the
+ * end of the launch.  All arguments are validated on the host first; a failed call launches
+ * nothing and writes nothing.  Returns SQUANT_OK or a negative SQUANT_ERR_* code.
+ */
+int squant_quantize_model(const squant_layer *layers, int32_t n_layers, const squant_options *opt,
+                          void *cuda_stream);
+
+/*
+ * The same, with HOST buffers: copies the weights to the current device, runs the grouped
+ * launch, copies codes / scales / error sums back and waits for the stream.  Device staging
+ * memory is cached inside the library between calls.  Pinned host memory gives the copies
+ * their full speed; pageable memory works.
+ */
+int squant_quantize_model_host(const squant_layer *layers, int32_t n_layers,
+                               const squant_options *opt, void *cuda_stream);
+
+/*
+ * Geometry of the launch that squant_quantize_model would issue for these descriptors
+ * (pointers are not dereferenced and may be NULL here).  Any output may be NULL.
+ */
+int squant_plan_info(const squant_layer *layers, int32_t n_layers, const squant_options *opt,
+                     int32_t *grid_ctas, int32_t *cta_threads, int32_t *dynamic_smem_bytes);
+
+/* Number of kernels this library has launched in this process (all entry points). */
+int64_t squant_launch_count(void);
+
+/* Human readable text for an error code; never NULL. */
+const char *squant_strerror(int code);
+
+/* Text of the CUDA error behind the calling thread's last SQUANT_ERR_CUDA ("" if none). */
+const char *squant_last_cuda_error(void);
+
+/* Frees cached plans and staging buffers on all devices.  Call with no work in flight. */
+int squant_shutdown(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SQUANT_H_ */

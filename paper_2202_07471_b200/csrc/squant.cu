@@ -1,0 +1,390 @@
+// Host side of the SQuant library: validation, launch plans, the C ABI of include/squant.h.
+#include "squant.h"
+
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <atomic>
+#include <cstdlib>
+#include <cstring>
+#include <list>
+#include <mutex>
+#include <string>
+#include <vector>
+
+#include "squant_device.cuh"
+
+namespace {
+
+using sq::Item;
+using sq::LayerDesc;
+
+constexpr int kMaxSmemFallback = 232448;   // 227 KB: per-CTA opt-in limit of sm_100
+constexpr int64_t kMaxChannelElems = 65535; // keeps the clamp-edge element out of every top-k
+                                            // (its perturbation is <= one ulp of qmax)
+constexpr size_t kMaxPlans = 16;
+
+std::mutex g_mutex;
+std::atomic<int64_t> g_launches{0};
+thread_local std::string t_cuda_error;
+
+int cuda_fail(cudaError_t e, const char *what)
+{
+    t_cuda_error = std::string(what) + ": " + cudaGetErrorString(e);
+    return SQUANT_ERR_CUDA;
+}
+
+#define SQ_CUDA(call)                                          \
+    do {                                                       \
+        cudaError_t e__ = (call);                              \
+        if (e__ != cudaSuccess) return cuda_fail(e__, #call);  \
+    } while (0)
+
+inline int align16(int v) { return (v + 15) & ~15; }
+
+struct HostPlan {
+    std::vector<LayerDesc> layers;
+    std::vector<Item> items;
+    int smem_bytes = 0;
+    int qmax = 0;
+    unsigned mode = 0;
+};
+
+// Threads that share one output channel, by channel length.
+int group_size(int64_t nk)
+{
+    if (nk <= 1024) return 32;
+    if (nk <= 2048) return 64;
+    if (nk <= 4096) return 128;
+    if (nk <= 8192) return 256;
+    return 512;
+}
+
+int validate(const squant_layer *layers, int32_t n_layers, const squant_options *opt,
+             bool need_pointers, squant_options &o)
+{
+    o.bits = 4;
+    o.mode = SQUANT_MODE_EKC;
+    o.flags = SQUANT_FLAG_NARROW_RANGE;
+    if (opt) {
+        o = *opt;
+        if (o.mode == 0) o.mode = SQUANT_MODE_EKC;
+    }
+    if (n_layers < 0) return SQUANT_ERR_SHAPE;
+    if (n_layers > 0 && !layers) return SQUANT_ERR_NULL;
+    if (o.bits < 2 || o.bits > 8) return SQUANT_ERR_BITS;
+    if (!(o.mode & SQUANT_MODE_E) || (o.mode & ~SQUANT_MODE_EKC)) return SQUANT_ERR_MODE;
+    if (o.flags & ~SQUANT_FLAG_NARROW_RANGE) return SQUANT_ERR_MODE;
+    for (int i = 0; i < n_layers; ++i) {
+        const squant_layer &l = layers[i];
+        if (l.cout <= 0 || l.cin <= 0 || l.kh <= 0 || l.kw <= 0) return SQUANT_ERR_SHAPE;
+        const int64_t k = static_cast<int64_t>(l.kh) * l.kw;
+        const int64_t nk = k * l.cin;
+        if (k > 65535 || nk > (1ll << 30)) return SQUANT_ERR_SHAPE;
+        if (static_cast<int64_t>(l.cout) * nk > (1ll << 40)) return SQUANT_ERR_SHAPE;
+        if (nk > kMaxChannelElems) return SQUANT_ERR_TOO_WIDE;
+        // E|C without K on kernels larger than 1x1 makes every element a channel candidate;
+        // that selection is not built.
+        if ((o.mode & SQUANT_MODE_C) && !(o.mode & SQUANT_MODE_K) && k > 1) return SQUANT_ERR_MODE;
+        if (need_pointers) {
+            if (!l.w || !l.codes || !l.scales) return SQUANT_ERR_NULL;
+            if ((reinterpret_cast<uintptr_t>(l.w) & 3) || (reinterpret_cast<uintptr_t>(l.scales) & 3) ||
+                (reinterpret_cast<uintptr_t>(l.kernel_err) & 3) ||
+                (reinterpret_cast<uintptr_t>(l.channel_err) & 3))
+                return SQUANT_ERR_ALIGN;
+        }
+    }
+    return SQUANT_OK;
+}
+
+// Shared-memory slice of one channel group and the grouped work list.
+int build_plan(const squant_layer *layers, int32_t n_layers, const squant_options &o, int max_smem,
+               HostPlan &p)
+{
+    p.qmax = (1 << (o.bits - 1)) - 1;
+    p.mode = o.mode;
+    p.layers.resize(n_layers);
+    p.smem_bytes = 0;
+    struct Batch { int64_t work; int layer; int ch0; };
+    std::vector<Batch> batches;
+    for (int i = 0; i < n_layers; ++i) {
+        const squant_layer &l = layers[i];
+        LayerDesc &d = p.layers[i];
+        d.w = l.w; d.codes = l.codes; d.scales = l.scales; d.kerr = l.kernel_err; d.cerr = l.channel_err;
+        d.M = l.cout; d.N = l.cin; d.K = l.kh * l.kw; d.NK = d.N * d.K;
+        d.g = group_size(d.NK);
+        d.g_shift = 0;
+        while ((1 << d.g_shift) < d.g) ++d.g_shift;
+        int off = align16(4 * d.NK);              // staged weights
+        d.off_codes = off; off += align16(d.NK);  // staged codes
+        if (d.K == 1) {                           // 1x1: perturbations overwrite the weights
+            d.off_ev = 0; d.off_vv = 0; d.off_vi = 0;
+        } else {
+            d.off_ev = off; off += align16(4 * d.N);
+            d.off_vv = off; off += align16(4 * d.N);
+            d.off_vi = off; off += align16(2 * d.N);
+        }
+        d.off_hist = off; off += 4 * sq::kHistBins;
+        d.off_red = off; off += 256;
+        d.slice_bytes = off;
+        const int groups = sq::kCtaThreads / d.g;
+        const int64_t cta_smem = static_cast<int64_t>(groups) * off;
+        if (cta_smem > max_smem) return SQUANT_ERR_TOO_WIDE;
+        if (cta_smem > p.smem_bytes) p.smem_bytes = static_cast<int>(cta_smem);
+        for (int c = 0; c < d.M; c += groups) {
+            const int nch = (d.M - c < groups) ? d.M - c : groups;
+            batches.push_back({static_cast<int64_t>(nch) * d.NK, i, c});
+        }
+    }
+    // Heaviest CTAs first, so that the tail of the launch is made of light ones.
+    std::stable_sort(batches.begin(), batches.end(),
+                     [](const Batch &a, const Batch &b) { return a.work > b.work; });
+    p.items.resize(batches.size());
+    for (size_t i = 0; i < batches.size(); ++i) p.items[i] = {batches[i].layer, batches[i].ch0};
+    return SQUANT_OK;
+}
+
+// A plan resident on one device, keyed by the exact descriptors and options.
+struct DevicePlan {
+    int device = -1;
+    std::string key;
+    void *table = nullptr;   // LayerDesc[n_layers] followed by Item[n_items]
+    int n_layers = 0, n_items = 0, smem_bytes = 0, qmax = 0;
+    unsigned mode = 0;
+};
+
+std::list<DevicePlan> g_plans;              // most recently used first
+std::vector<int> g_smem_limit_by_device;   // opt-in limit set on the kernel, per device
+
+std::string plan_key(const squant_layer *layers, int32_t n_layers, const squant_options &o)
+{
+    std::string k(reinterpret_cast<const char *>(&o), sizeof(o));
+    k.append(reinterpret_cast<const char *>(layers), sizeof(squant_layer) * static_cast<size_t>(n_layers));
+    return k;
+}
+
+int device_smem_limit(int device, int &limit)
+{
+    if (static_cast<int>(g_smem_limit_by_device.size()) <= device)
+        g_smem_limit_by_device.resize(device + 1, 0);
+    if (g_smem_limit_by_device[device] == 0) {
+        int v = 0;
+        SQ_CUDA(cudaDeviceGetAttribute(&v, cudaDevAttrMaxSharedMemoryPerBlockOptin, device));
+        SQ_CUDA(cudaFuncSetAttribute(sq::squant_model_kernel,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, v));
+        g_smem_limit_by_device[device] = v;
+    }
+    limit = g_smem_limit_by_device[device];
+    return SQUANT_OK;
+}
+
+int get_plan(const squant_layer *layers, int32_t n_layers, const squant_options &o,
+             cudaStream_t stream, DevicePlan *&out)
+{
+    int device = 0;
+    SQ_CUDA(cudaGetDevice(&device));
+    std::string key = plan_key(layers, n_layers, o);
+    for (auto it = g_plans.begin(); it != g_plans.end(); ++it) {
+        if (it->device == device && it->key == key) {
+            g_plans.splice(g_plans.begin(), g_plans, it);
+            out = &g_plans.front();
+            return SQUANT_OK;
+        }
+    }
+    int limit = 0;
+    int rc = device_smem_limit(device, limit);
+    if (rc) return rc;
+    HostPlan hp;
+    rc = build_plan(layers, n_layers, o, limit, hp);
+    if (rc) return rc;
+    DevicePlan dp;
+    dp.device = device;
+    dp.key = std::move(key);
+    dp.n_layers = n_layers;
+    dp.n_items = static_cast<int>(hp.items.size());
+    dp.smem_bytes = hp.smem_bytes;
+    dp.qmax = hp.qmax;
+    dp.mode = hp.mode;
+    const size_t lbytes = sizeof(LayerDesc) * hp.layers.size();
+    const size_t ibytes = sizeof(Item) * hp.items.size();
+    if (lbytes + ibytes > 0) {
+        std::vector<unsigned char> host(lbytes + ibytes);
+        std::memcpy(host.data(), hp.layers.data(), lbytes);
+        std::memcpy(host.data() + lbytes, hp.items.data(), ibytes);
+        cudaError_t e = cudaMalloc(&dp.table, lbytes + ibytes);
+        if (e != cudaSuccess) return e == cudaErrorMemoryAllocation ? SQUANT_ERR_NOMEM : cuda_fail(e, "cudaMalloc");
+        e = cudaMemcpyAsync(dp.table, host.data(), lbytes + ibytes, cudaMemcpyHostToDevice, stream);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(stream);   // host vector dies here
+        if (e != cudaSuccess) { cudaFree(dp.table); return cuda_fail(e, "plan upload"); }
+    }
+    if (g_plans.size() >= kMaxPlans) {
+        // The evicted table may still be read by an earlier launch: wait for the device first.
+        int cur = device;
+        cudaSetDevice(g_plans.back().device);
+        cudaDeviceSynchronize();
+        cudaFree(g_plans.back().table);
+        cudaSetDevice(cur);
+        g_plans.pop_back();
+    }
+    g_plans.push_front(std::move(dp));
+    out = &g_plans.front();
+    return SQUANT_OK;
+}
+
+int launch_plan(const DevicePlan &dp, cudaStream_t stream)
+{
+    if (dp.n_items == 0) return SQUANT_OK;
+    const LayerDesc *dl = static_cast<const LayerDesc *>(dp.table);
+    const Item *di = reinterpret_cast<const Item *>(static_cast<const unsigned char *>(dp.table) +
+                                                    sizeof(LayerDesc) * dp.n_layers);
+    sq::squant_model_kernel<<<dp.n_items, sq::kCtaThreads, dp.smem_bytes, stream>>>(dl, di, dp.qmax, dp.mode);
+    SQ_CUDA(cudaGetLastError());
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return SQUANT_OK;
+}
+
+// Device staging of the host-buffer entry point, one arena per device, grown on demand.
+struct Arena { void *ptr = nullptr; size_t bytes = 0; };
+std::vector<Arena> g_arenas;
+
+inline size_t align256(size_t v) { return (v + 255) & ~static_cast<size_t>(255); }
+
+}  // namespace
+
+extern "C" {
+
+int squant_quantize_model(const squant_layer *layers, int32_t n_layers, const squant_options *opt,
+                          void *cuda_stream)
+{
+    squant_options o;
+    int rc = validate(layers, n_layers, opt, true, o);
+    if (rc) return rc;
+    if (n_layers == 0) return SQUANT_OK;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    DevicePlan *dp = nullptr;
+    rc = get_plan(layers, n_layers, o, static_cast<cudaStream_t>(cuda_stream), dp);
+    if (rc) return rc;
+    return launch_plan(*dp, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int squant_quantize_layer(const squant_layer *layer, const squant_options *opt, void *cuda_stream)
+{
+    if (!layer) return SQUANT_ERR_NULL;
+    return squant_quantize_model(layer, 1, opt, cuda_stream);
+}
+
+int squant_quantize_model_host(const squant_layer *layers, int32_t n_layers,
+                               const squant_options *opt, void *cuda_stream)
+{
+    squant_options o;
+    int rc = validate(layers, n_layers, opt, true, o);
+    if (rc) return rc;
+    if (n_layers == 0) return SQUANT_OK;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    std::lock_guard<std::mutex> lock(g_mutex);
+    int device = 0;
+    SQ_CUDA(cudaGetDevice(&device));
+    // carve one device arena: per layer weights, codes, scales, kernel sums, channel sums
+    std::vector<squant_layer> dev(layers, layers + n_layers);
+    std::vector<size_t> off(static_cast<size_t>(n_layers) * 5);
+    size_t total = 0;
+    for (int i = 0; i < n_layers; ++i) {
+        const squant_layer &l = layers[i];
+        const size_t n = static_cast<size_t>(l.cin) * l.kh * l.kw * l.cout;
+        off[5 * i + 0] = total; total += align256(n * 4);
+        off[5 * i + 1] = total; total += align256(n);
+        off[5 * i + 2] = total; total += align256(static_cast<size_t>(l.cout) * 4);
+        off[5 * i + 3] = total; total += l.kernel_err ? align256(static_cast<size_t>(l.cout) * l.cin * 4) : 0;
+        off[5 * i + 4] = total; total += l.channel_err ? align256(static_cast<size_t>(l.cout) * 4) : 0;
+    }
+    if (static_cast<int>(g_arenas.size()) <= device) g_arenas.resize(device + 1);
+    Arena &a = g_arenas[device];
+    if (a.bytes < total) {
+        if (a.ptr) { SQ_CUDA(cudaDeviceSynchronize()); SQ_CUDA(cudaFree(a.ptr)); a.ptr = nullptr; a.bytes = 0; }
+        cudaError_t e = cudaMalloc(&a.ptr, total);
+        if (e != cudaSuccess) { a.ptr = nullptr; return e == cudaErrorMemoryAllocation ? SQUANT_ERR_NOMEM : cuda_fail(e, "cudaMalloc"); }
+        a.bytes = total;
+    }
+    unsigned char *base = static_cast<unsigned char *>(a.ptr);
+    for (int i = 0; i < n_layers; ++i) {
+        const squant_layer &l = layers[i];
+        const size_t n = static_cast<size_t>(l.cin) * l.kh * l.kw * l.cout;
+        dev[i].w = reinterpret_cast<const float *>(base + off[5 * i + 0]);
+        dev[i].codes = reinterpret_cast<int8_t *>(base + off[5 * i + 1]);
+        dev[i].scales = reinterpret_cast<float *>(base + off[5 * i + 2]);
+        dev[i].kernel_err = l.kernel_err ? reinterpret_cast<float *>(base + off[5 * i + 3]) : nullptr;
+        dev[i].channel_err = l.channel_err ? reinterpret_cast<float *>(base + off[5 * i + 4]) : nullptr;
+        SQ_CUDA(cudaMemcpyAsync(base + off[5 * i + 0], l.w, n * 4, cudaMemcpyHostToDevice, stream));
+    }
+    DevicePlan *dp = nullptr;
+    rc = get_plan(dev.data(), n_layers, o, stream, dp);
+    if (rc) return rc;
+    rc = launch_plan(*dp, stream);
+    if (rc) return rc;
+    for (int i = 0; i < n_layers; ++i) {
+        const squant_layer &l = layers[i];
+        const size_t n = static_cast<size_t>(l.cin) * l.kh * l.kw * l.cout;
+        SQ_CUDA(cudaMemcpyAsync(l.codes, dev[i].codes, n, cudaMemcpyDeviceToHost, stream));
+        SQ_CUDA(cudaMemcpyAsync(l.scales, dev[i].scales, static_cast<size_t>(l.cout) * 4, cudaMemcpyDeviceToHost, stream));
+        if (l.kernel_err)
+            SQ_CUDA(cudaMemcpyAsync(l.kernel_err, dev[i].kernel_err, static_cast<size_t>(l.cout) * l.cin * 4, cudaMemcpyDeviceToHost, stream));
+        if (l.channel_err)
+            SQ_CUDA(cudaMemcpyAsync(l.channel_err, dev[i].channel_err, static_cast<size_t>(l.cout) * 4, cudaMemcpyDeviceToHost, stream));
+    }
+    SQ_CUDA(cudaStreamSynchronize(stream));
+    return SQUANT_OK;
+}
+
+int squant_plan_info(const squant_layer *layers, int32_t n_layers, const squant_options *opt,
+                     int32_t *grid_ctas, int32_t *cta_threads, int32_t *dynamic_smem_bytes)
+{
+    squant_options o;
+    int rc = validate(layers, n_layers, opt, false, o);
+    if (rc) return rc;
+    HostPlan hp;
+    rc = build_plan(layers, n_layers, o, kMaxSmemFallback, hp);
+    if (rc) return rc;
+    if (grid_ctas) *grid_ctas = static_cast<int32_t>(hp.items.size());
+    if (cta_threads) *cta_threads = sq::kCtaThreads;
+    if (dynamic_smem_bytes) *dynamic_smem_bytes = hp.smem_bytes;
+    return SQUANT_OK;
+}
+
+int64_t squant_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char *squant_strerror(int code)
+{
+    switch (code) {
+        case SQUANT_OK: return "success";
+        case SQUANT_ERR_NULL: return "a required pointer is NULL";
+        case SQUANT_ERR_SHAPE: return "a layer dimension is not positive or the element count overflows";
+        case SQUANT_ERR_BITS: return "bits must be in 2..8";
+        case SQUANT_ERR_MODE: return "mode mask must contain E and be one of E, E|K, E|K|C (E|C only for 1x1 kernels); unknown flag bits are rejected";
+        case SQUANT_ERR_ALIGN: return "float pointers must be 4-byte aligned";
+        case SQUANT_ERR_TOO_WIDE: return "an output channel (cin*kh*kw) does not fit the on-chip path";
+        case SQUANT_ERR_CUDA: return "a CUDA runtime call failed (see squant_last_cuda_error)";
+        case SQUANT_ERR_NOMEM: return "out of host or device memory";
+        default: return "unknown squant error code";
+    }
+}
+
+const char *squant_last_cuda_error(void) { return t_cuda_error.c_str(); }
+
+int squant_shutdown(void)
+{
+    std::lock_guard<std::mutex> lock(g_mutex);
+    int cur = 0;
+    const bool have = cudaGetDevice(&cur) == cudaSuccess;
+    for (auto &p : g_plans) {
+        if (p.table) { cudaSetDevice(p.device); cudaDeviceSynchronize(); cudaFree(p.table); }
+    }
+    g_plans.clear();
+    for (size_t d = 0; d < g_arenas.size(); ++d) {
+        if (g_arenas[d].ptr) { cudaSetDevice(static_cast<int>(d)); cudaDeviceSynchronize(); cudaFree(g_arenas[d].ptr); }
+    }
+    g_arenas.clear();
+    if (have) cudaSetDevice(cur);
+    return SQUANT_OK;
+}
+
+}  // extern "C"

@@ -173,25 +173,50 @@ def _fill(recipe: str, key: int, start: int, count: int, std: float) -> np.ndarr
     raise ValueError(f"unknown recipe {recipe!r}")
 
 
-def layer_weights(wl: Workload, layer: int, seed: int = 0, *, channels: slice | None = None,
-                  chunk: int = 1 << 22) -> np.ndarray:
-    """fp32 weights of one layer, shape [cout, cin, kh, kw] (or the selected channel range)."""
+def _fill_channels(wl: Workload, layer: int, seed: int, c0: int, c1: int, out: np.ndarray,
+                   chunk: int) -> None:
+    """Write channels c0..c1-1 of one layer into out[(c1-c0) * per_ch] (flat fp32)."""
     m, n, kh, kw = wl.shapes[layer]
     per_ch = n * kh * kw
-    c0, c1, _ = (channels or slice(None)).indices(m)
     key = stream_key(wl.config_id, seed, layer)
     std = _fan_in_std(wl.shapes[layer])
-    out = np.empty((c1 - c0) * per_ch, dtype=np.float32)
     lo, hi = c0 * per_ch, c1 * per_ch
     for s in range(lo, hi, chunk):
         e = min(hi, s + chunk)
         out[s - lo:e - lo] = _fill(wl.recipe, key, s, e - s, std).astype(np.float32)
-    out = out.reshape(c1 - c0, n, kh, kw)
     if wl.recipe == "normal_chanscale":
         u = uniform01(stream_key(key, 4), c0, c1 - c0)
         mult = np.exp(math.log(0.5) + u * (math.log(2.0) - math.log(0.5)))
-        out *= mult.astype(np.float32)[:, None, None, None]
-    return out
+        out.reshape(c1 - c0, per_ch)[...] *= mult.astype(np.float32)[:, None]
+
+
+def layer_weights(wl: Workload, layer: int, seed: int = 0, *, channels: slice | None = None,
+                  chunk: int = 1 << 20, threads: int = 1, out: np.ndarray | None = None) -> np.ndarray:
+    """fp32 weights of one layer, shape [cout, cin, kh, kw] (or the selected channel range).
+
+    Values depend only on (workload, layer, seed, position): any channel range, chunk size or
+    thread count gives the same numbers.  `out` may be a preallocated fp32 array to fill."""
+    m, n, kh, kw = wl.shapes[layer]
+    per_ch = n * kh * kw
+    c0, c1, _ = (channels or slice(None)).indices(m)
+    if out is None:
+        out = np.empty((c1 - c0, n, kh, kw), dtype=np.float32)
+    flat = out.reshape(-1)
+    assert flat.size == (c1 - c0) * per_ch and flat.dtype == np.float32
+    threads = max(1, min(int(threads), c1 - c0))
+    if threads == 1:
+        _fill_channels(wl, layer, seed, c0, c1, flat, chunk)
+    else:
+        from concurrent.futures import ThreadPoolExecutor
+        n_parts = min(c1 - c0, threads * 4)
+        edges = [c0 + (c1 - c0) * i // n_parts for i in range(n_parts + 1)]
+        with ThreadPoolExecutor(threads) as pool:
+            futs = [pool.submit(_fill_channels, wl, layer, seed, a, b,
+                                flat[(a - c0) * per_ch:(b - c0) * per_ch], chunk)
+                    for a, b in zip(edges[:-1], edges[1:]) if b > a]
+            for f in futs:
+                f.result()
+    return out.reshape(c1 - c0, n, kh, kw)
 
 
 def iter_layers(wl: Workload, seed: int = 0) -> Iterator[Tuple[int, Shape, np.ndarray]]:

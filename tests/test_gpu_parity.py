@@ -1,0 +1,154 @@
+"""CUDA path vs the CPU checker, element by element, through the C ABI (needs a B200)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2202_07471_b200 as sq
+from paper_2202_07471_b200 import workloads as W
+
+from cases import SWEEP_SHAPES, adversarial_layer, coarse
+
+pytestmark = pytest.mark.gpu
+
+E, EK, EKC = sq.MODE_E, sq.MODE_E | sq.MODE_K, sq.MODE_EKC
+
+
+def run_gpu(ws, bits, mode, flags=sq.FLAG_NARROW_RANGE):
+    """Quantize a list of numpy layers in one grouped launch; returns LayerBuffers on the host."""
+    bufs = [sq.alloc_outputs(torch.from_numpy(np.ascontiguousarray(w)).cuda()) for w in ws]
+    for b in bufs:   # poison the outputs so that an unwritten element cannot pass
+        b.codes.fill_(-128); b.scales.fill_(float("nan")); b.kernel_err.fill_(float("nan")); b.channel_err.fill_(float("nan"))
+    sq.squant_quantize_model(bufs, bits=bits, mode=mode, flags=flags)
+    torch.cuda.synchronize()
+    return bufs
+
+
+def assert_layer_equal(b, w, bits, mode, flags=oracle.FLAG_NARROW_RANGE, tag=""):
+    r = oracle.quantize_layer(w, bits=bits, mode=mode, flags=flags)
+    codes = b.codes.cpu().numpy()
+    bad = np.argwhere(codes != r.codes)
+    assert bad.size == 0, f"{tag}: {len(bad)} codes differ, first at {bad[0].tolist()}"
+    # bit-exact floats: compare the raw words
+    assert np.array_equal(b.scales.cpu().numpy().view(np.uint32), r.scales.view(np.uint32)), f"{tag}: scales"
+    assert np.array_equal(b.kernel_err.cpu().numpy().view(np.uint32), r.kernel_err.view(np.uint32)), f"{tag}: kernel_err"
+    assert np.array_equal(b.channel_err.cpu().numpy().view(np.uint32), r.channel_err.view(np.uint32)), f"{tag}: channel_err"
+
+
+def test_single_conv_config():
+    """Config 1: one [64,64,3,3] layer, N(0, sqrt(2/576)), seed 0, 4 bit, E+K+C."""
+    w = W.layer_weights(W.WORKLOADS["single_conv"], 0, seed=0)
+    for mode in (E, EK, EKC):
+        (b,) = run_gpu([w], 4, mode)
+        assert_layer_equal(b, w, 4, mode, tag=f"mode{mode}")
+
+
+@pytest.mark.parametrize("bits", [2, 3, 4, 6, 8])
+def test_shape_sweep_grouped(bits):
+    """Every sweep shape in ONE grouped launch: ragged tails, every kernel size path, all group
+    sizes, special channels (zero, constant, tiny, huge, ties)."""
+    ws = [adversarial_layer(s, seed=17 * bits + i) for i, s in enumerate(SWEEP_SHAPES)]
+    for mode in (EKC, EK, E):
+        bufs = run_gpu(ws, bits, mode)
+        for i, (b, w) in enumerate(zip(bufs, ws)):
+            assert_layer_equal(b, w, bits, mode, tag=f"shape{SWEEP_SHAPES[i]} mode{mode}")
+
+
+def test_e_c_mode_on_1x1():
+    ws = [adversarial_layer(s, seed=5) for s in [(7, 300, 1, 1), (4, 2049, 1, 1)]]
+    mode = sq.MODE_E | sq.MODE_C
+    bufs = run_gpu(ws, 4, mode)
+    for b, w in zip(bufs, ws):
+        assert_layer_equal(b, w, 4, mode)
+
+
+def test_wide_range_flag():
+    w = adversarial_layer((16, 40, 3, 3), seed=2)
+    (b,) = run_gpu([w], 4, EKC, flags=0)
+    assert_layer_equal(b, w, 4, EKC, flags=0)
+
+
+def test_unaligned_views_and_null_optional_outputs():
+    """Weights and codes that start off a 16-byte boundary take the scalar load/store path."""
+    w = adversarial_layer((6, 37, 3, 3), seed=8)
+    n = w.size
+    base = torch.zeros(n + 3, dtype=torch.float32, device="cuda")
+    cbase = torch.full((n + 5,), -128, dtype=torch.int8, device="cuda")
+    wv = base[3:3 + n].view(w.shape)
+    wv.copy_(torch.from_numpy(w))
+    b = sq.LayerBuffers(wv, cbase[5:5 + n].view(w.shape), torch.empty(6, device="cuda"), None, None)
+    sq.squant_quantize_model([b], bits=4)
+    torch.cuda.synchronize()
+    r = oracle.quantize_layer(w, bits=4)
+    assert np.array_equal(b.codes.cpu().numpy(), r.codes)
+    assert np.array_equal(b.scales.cpu().numpy(), r.scales)
+    assert int(cbase[:5].max()) == -128
+
+
+def test_coarse_grid_ties_large_channel():
+    """Heavy ties in both selections on a full-width channel (radix select must fall through
+    to the index digits)."""
+    w = coarse(W.random_layer((3, 2048, 3, 3), seed=1), steps=24, div=4)
+    (b,) = run_gpu([w], 4, EKC)
+    assert_layer_equal(b, w, 4, EKC)
+    w = np.full((2, 1500, 3, 3), 0.3, dtype=np.float32)
+    w[:, 0, 0, 0] = 1.0
+    (b,) = run_gpu([w], 8, EKC)
+    assert_layer_equal(b, w, 8, EKC)
+
+
+@pytest.mark.parametrize("name,bits", [("resnet18", 4), ("resnet50", 4), ("resnet50", 6), ("mobilenetv2", 4)])
+def test_model_configs_full(name, bits):
+    """Configs 2-4 at full size, the whole model in one grouped launch, every element compared."""
+    wl = W.WORKLOADS[name]
+    ws = [W.layer_weights(wl, i, seed=0, threads=8) for i in range(len(wl.shapes))]
+    bufs = run_gpu(ws, bits, EKC)
+    for i, (b, w) in enumerate(zip(bufs, ws)):
+        assert_layer_equal(b, w, bits, EKC, tag=f"{name} layer {i} {wl.shapes[i]}")
+
+
+def test_large_layer_config_sampled():
+    """Config 5 at full size (8 x [2048,2048,3,3]) in the launch configuration the benchmark
+    times; the checker recomputes a sample of whole output channels (channels are independent
+    sub-problems), and properties that hold at any size are checked on everything."""
+    wl = W.WORKLOADS["large_layer"]
+    host = [torch.empty(s, dtype=torch.float32).pin_memory() for s in wl.shapes]
+    for i, t in enumerate(host):
+        W.layer_weights(wl, i, seed=0, threads=8, out=t.numpy())
+    bufs = [sq.alloc_outputs(t.cuda()) for t in host]
+    sq.squant_quantize_model(bufs, bits=4, mode=EKC)
+    torch.cuda.synchronize()
+    for i, b in enumerate(bufs):
+        assert int(b.codes.abs().max()) <= 7
+        assert float(b.channel_err.abs().max()) <= 0.5          # Eq. 11
+        assert float(b.kernel_err.abs().max()) <= 1.0           # r_k = 1.0 after SQuant-C
+        tot = b.kernel_err.double().sum(1)
+        assert float((tot - b.channel_err.double()).abs().max()) < 1e-3
+        pick = np.arange(i, 2048, 61)
+        w = host[i].numpy()[pick]
+        r = oracle.quantize_layer(w, bits=4, mode=EKC)
+        assert np.array_equal(b.codes[pick].cpu().numpy(), r.codes), f"layer {i}"
+        assert np.array_equal(b.scales[pick].cpu().numpy(), r.scales)
+        assert np.array_equal(b.kernel_err[pick].cpu().numpy(), r.kernel_err)
+        assert np.array_equal(b.channel_err[pick].cpu().numpy(), r.channel_err)
+
+
+def test_host_entry_point_matches_device_entry_point():
+    wl = W.WORKLOADS["single_conv"]
+    w = W.layer_weights(wl, 0)
+    hb = sq.alloc_outputs(torch.from_numpy(w).pin_memory(), pin=True)
+    sq.squant_quantize_model_host([hb], bits=4)
+    r = oracle.quantize_layer(w, bits=4)
+    assert np.array_equal(hb.codes.numpy(), r.codes) and np.array_equal(hb.scales.numpy(), r.scales)
+    assert np.array_equal(hb.kernel_err.numpy(), r.kernel_err)
+    assert np.array_equal(hb.channel_err.numpy(), r.channel_err)
+
+
+def test_repeat_calls_are_deterministic_and_counted():
+    w = torch.from_numpy(W.random_layer((32, 64, 3, 3), 3)).cuda()
+    n0 = sq.squant_launch_count()
+    a = sq.squant_quantize_layer(w, bits=4)
+    b = sq.squant_quantize_layer(w, bits=4)
+    torch.cuda.synchronize()
+    assert sq.squant_launch_count() == n0 + 2
+    assert torch.equal(a.codes, b.codes) and torch.equal(a.kernel_err, b.kernel_err)
