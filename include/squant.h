@@ -62,6 +62,8 @@ extern "C" {
 #define SQUANT_ERR_TOO_WIDE (-6)    /* one output channel does not fit the on-chip path */
 #define SQUANT_ERR_CUDA (-7)        /* a CUDA runtime call failed; see squant_last_cuda_error() */
 #define SQUANT_ERR_NOMEM (-8)       /* host or device allocation failed */
+#define SQUANT_ERR_LIMIT (-9)       /* the layer needs more launch-table entries than the fixed
+                                       table of squant_quantize_layer_noalloc holds */
 
 typedef struct squant_options {
     int32_t bits;   /* 2..8; qmax = 2^(bits-1) - 1 */
@@ -123,6 +125,46 @@ int squant_quantize_model_host(const squant_layer *layers, int32_t n_layers,
  */
 int squant_plan_info(const squant_layer *layers, int32_t n_layers, const squant_options *opt,
                      int32_t *grid_ctas, int32_t *cta_threads, int32_t *dynamic_smem_bytes);
+
+/*
+ * squant_quantize_layer without any device allocation.  (An addition of this library; the paper
+ * has no counterpart.)
+ *
+ * Who needs it: code that must not call cudaMalloc while it runs - a serving or training process
+ * whose framework has handed every free byte of the GPU to its own memory pool (cudaMalloc then
+ * fails or fragments the pool), a latency-critical loop that cannot take the device-wide
+ * synchronisation cudaMalloc / cudaFree imply, or a host that is only allowed to run
+ * pre-loaded code.  squant_quantize_layer and squant_quantize_model keep their launch table
+ * (layer descriptor + one entry per CTA) in cudaMalloc'ed memory; this entry point keeps it in
+ * a fixed array that is part of the library image instead, so it calls no cudaMalloc, cudaFree
+ * or other allocating routine.  Every GPU that loads the library holds that array
+ * (SQUANT_NOALLOC_TABLE_BYTES, about 256 KB) until the process exits.
+ *
+ *   layer, opt, cuda_stream   as for squant_quantize_layer; DEVICE pointers, caller-owned
+ *
+ * Limits: one layer per call, and the layer's launch must need at most SQUANT_NOALLOC_MAX_CTAS
+ * thread blocks (one block handles 512/g output channels, g = 32..512 threads per channel by
+ * channel length; squant_plan_info reports the count).  A larger layer is rejected with
+ * SQUANT_ERR_LIMIT before anything is launched; split it by output-channel range and call once
+ * per part.
+ *
+ * Sharing: all calls on a device use the same table, and each call overwrites the part it
+ * needs (nothing in it has to start at zero; the previous call's entries beyond that part are
+ * left behind and never read).  Calls are ordered correctly when they are issued to the same
+ * stream.  Two calls whose GPU work can overlap - different streams without an event between
+ * them - race: the second call's table upload may land while the first call's kernel is still
+ * reading it.  Serialise such calls.
+ *
+ * The first call on each device looks up the table's device address and raises the kernel's
+ * shared-memory limit; make that first call outside any stream capture.
+ *
+ * Results are bit-identical to squant_quantize_layer.  Returns SQUANT_OK or a negative
+ * SQUANT_ERR_* code; a failed call launches nothing and writes nothing.
+ */
+#define SQUANT_NOALLOC_MAX_CTAS 32768
+#define SQUANT_NOALLOC_TABLE_BYTES (256 + 8 * SQUANT_NOALLOC_MAX_CTAS)
+int squant_quantize_layer_noalloc(const squant_layer *layer, const squant_options *opt,
+                                  void *cuda_stream);
 
 /* Number of kernels this library has launched in this process (all entry points). */
 int64_t squant_launch_count(void);

@@ -19,7 +19,9 @@ FLAG_NARROW_RANGE = 1
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libsquant.so")
 
-EXPORTS = ("squant_quantize_layer", "squant_quantize_model", "squant_quantize_model_host",
+NOALLOC_MAX_CTAS = 32768
+
+EXPORTS = ("squant_quantize_layer", "squant_quantize_layer_noalloc", "squant_quantize_model", "squant_quantize_model_host",
            "squant_plan_info", "squant_launch_count", "squant_strerror", "squant_last_cuda_error",
            "squant_shutdown")
 
@@ -56,10 +58,11 @@ def load_library() -> ctypes.CDLL:
     lib = ctypes.CDLL(LIB_PATH)
     lp, op, vp, i32p = ctypes.POINTER(Layer), ctypes.POINTER(Options), ctypes.c_void_p, ctypes.POINTER(ctypes.c_int32)
     lib.squant_quantize_layer.argtypes = [lp, op, vp]
+    lib.squant_quantize_layer_noalloc.argtypes = [lp, op, vp]
     lib.squant_quantize_model.argtypes = [lp, ctypes.c_int32, op, vp]
     lib.squant_quantize_model_host.argtypes = [lp, ctypes.c_int32, op, vp]
     lib.squant_plan_info.argtypes = [lp, ctypes.c_int32, op, i32p, i32p, i32p]
-    for f in ("squant_quantize_layer", "squant_quantize_model", "squant_quantize_model_host",
+    for f in ("squant_quantize_layer", "squant_quantize_layer_noalloc", "squant_quantize_model", "squant_quantize_model_host",
               "squant_plan_info", "squant_shutdown"):
         getattr(lib, f).restype = ctypes.c_int
     lib.squant_launch_count.restype = ctypes.c_int64
@@ -175,6 +178,25 @@ def squant_quantize_layer(w: torch.Tensor, bits: int = 4, mode: int = MODE_EKC,
     opt = _options(bits, mode, flags)
     _check(load_library().squant_quantize_layer(ctypes.byref(d), ctypes.byref(opt), _stream_handle(stream)))
     return b
+
+
+def squant_quantize_layer_noalloc(buffers: LayerBuffers, bits: int = 4, mode: int = MODE_EKC,
+                                  flags: int = FLAG_NARROW_RANGE,
+                                  stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Quantize one layer into caller-provided CUDA tensors without any device allocation.
+
+    For callers that must not allocate GPU memory while running (a framework pool owns the
+    device, or the allocation's device-wide synchronisation is not acceptable): the launch table
+    lives in a fixed array inside the library.  One layer per call, at most NOALLOC_MAX_CTAS
+    thread blocks (SquantError code -9 beyond that), and calls whose GPU work may overlap must be
+    serialised by the caller because they share that array.  This wrapper itself creates no
+    tensors; results equal squant_quantize_layer bit for bit."""
+    if not buffers.w.is_cuda:
+        raise ValueError("squant_quantize_layer_noalloc needs CUDA tensors")
+    d = _descriptor(buffers)
+    opt = _options(bits, mode, flags)
+    _check(load_library().squant_quantize_layer_noalloc(ctypes.byref(d), ctypes.byref(opt),
+                                                        _stream_handle(stream)))
 
 
 def squant_plan_info(shapes: Sequence[Sequence[int]], bits: int = 4, mode: int = MODE_EKC,

@@ -249,6 +249,28 @@ std::vector<Arena> g_arenas;
 
 inline size_t align256(size_t v) { return (v + 255) & ~static_cast<size_t>(255); }
 
+// ---- launch table of squant_quantize_layer_noalloc: part of the library image, never allocated.
+// Layout: one LayerDesc in the first 256 bytes, then up to SQUANT_NOALLOC_MAX_CTAS Items.
+// In host code the name below is only a handle of the symbol; the address a kernel can use comes
+// from cudaGetSymbolAddress, taken once per device with that device current.
+static_assert(sizeof(LayerDesc) <= 256, "layer descriptor must fit the table header");
+static_assert(sizeof(Item) == 8, "table size in squant.h assumes 8-byte entries");
+static __device__ __align__(256) unsigned char g_noalloc_table[SQUANT_NOALLOC_TABLE_BYTES];
+unsigned char g_noalloc_host[SQUANT_NOALLOC_TABLE_BYTES];   // host image, guarded by g_mutex
+std::vector<void *> g_noalloc_dev;                          // per device: address of the table
+
+int noalloc_table_address(int device, void *&ptr)
+{
+    if (static_cast<int>(g_noalloc_dev.size()) <= device) g_noalloc_dev.resize(device + 1, nullptr);
+    if (!g_noalloc_dev[device]) {
+        void *p = nullptr;
+        SQ_CUDA(cudaGetSymbolAddress(&p, g_noalloc_table));   // current device is `device`
+        g_noalloc_dev[device] = p;
+    }
+    ptr = g_noalloc_dev[device];
+    return SQUANT_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -335,6 +357,43 @@ int squant_quantize_model_host(const squant_layer *layers, int32_t n_layers,
     return SQUANT_OK;
 }
 
+int squant_quantize_layer_noalloc(const squant_layer *layer, const squant_options *opt,
+                                  void *cuda_stream)
+{
+    if (!layer) return SQUANT_ERR_NULL;
+    squant_options o;
+    int rc = validate(layer, 1, opt, true, o);
+    if (rc) return rc;
+    HostPlan hp;   // host-side bookkeeping only; nothing below allocates device memory
+    rc = build_plan(layer, 1, o, kMaxSmemFallback, hp);
+    if (rc) return rc;
+    if (hp.items.size() > static_cast<size_t>(SQUANT_NOALLOC_MAX_CTAS)) return SQUANT_ERR_LIMIT;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    std::lock_guard<std::mutex> lock(g_mutex);
+    int device = 0;
+    SQ_CUDA(cudaGetDevice(&device));
+    int limit = 0;
+    rc = device_smem_limit(device, limit);
+    if (rc) return rc;
+    if (hp.smem_bytes > limit) return SQUANT_ERR_TOO_WIDE;
+    void *table = nullptr;
+    rc = noalloc_table_address(device, table);
+    if (rc) return rc;
+    const size_t ibytes = sizeof(Item) * hp.items.size();
+    std::memcpy(g_noalloc_host, hp.layers.data(), sizeof(LayerDesc));
+    std::memcpy(g_noalloc_host + 256, hp.items.data(), ibytes);
+    // Pageable source: the runtime has taken its copy of the bytes when this returns, so the host
+    // image may be rewritten by the next call; the device-side copy is ordered on `stream`.
+    SQ_CUDA(cudaMemcpyAsync(table, g_noalloc_host, 256 + ibytes, cudaMemcpyHostToDevice, stream));
+    const LayerDesc *dl = static_cast<const LayerDesc *>(table);
+    const Item *di = reinterpret_cast<const Item *>(static_cast<const unsigned char *>(table) + 256);
+    sq::squant_model_kernel<<<static_cast<unsigned>(hp.items.size()), sq::kCtaThreads, hp.smem_bytes, stream>>>(
+        dl, di, hp.qmax, hp.mode);
+    SQ_CUDA(cudaGetLastError());
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return SQUANT_OK;
+}
+
 int squant_plan_info(const squant_layer *layers, int32_t n_layers, const squant_options *opt,
                      int32_t *grid_ctas, int32_t *cta_threads, int32_t *dynamic_smem_bytes)
 {
@@ -364,6 +423,7 @@ const char *squant_strerror(int code)
         case SQUANT_ERR_TOO_WIDE: return "an output channel (cin*kh*kw) does not fit the on-chip path";
         case SQUANT_ERR_CUDA: return "a CUDA runtime call failed (see squant_last_cuda_error)";
         case SQUANT_ERR_NOMEM: return "out of host or device memory";
+        case SQUANT_ERR_LIMIT: return "the layer needs more thread blocks than the fixed launch table of squant_quantize_layer_noalloc holds (SQUANT_NOALLOC_MAX_CTAS); split it by output-channel range";
         default: return "unknown squant error code";
     }
 }
