@@ -298,23 +298,156 @@ __device__ __forceinline__ int select_threshold(const Group &G, const int *vv, i
     return k_eff;
 }
 
-// ---------------------------------------------------------------- one output channel
-template <int KT>
-__device__ __forceinline__ void quantize_channel(const LayerDesc &L, int m, const Group &G,
-                                                 unsigned char *slice, int qmax, unsigned mode)
-{
-    const int K = KT ? KT : L.K;
-    const int N = L.N, NK = L.NK;
-    float *wbuf = reinterpret_cast<float *>(slice);
-    int8_t *cbuf = reinterpret_cast<int8_t *>(slice + L.off_codes);
-    int *ev = reinterpret_cast<int *>(slice + L.off_ev);
-    int *vv = reinterpret_cast<int *>(slice + L.off_vv);
-    unsigned short *vi = reinterpret_cast<unsigned short *>(slice + L.off_vi);
-    int *hist = reinterpret_cast<int *>(slice + L.off_hist);
-    unsigned char *red = slice + L.off_red;
-    int *bc = reinterpret_cast<int *>(red + 128);
+// ---------------------------------------------------------------- 3x3 fast path
+// The division w / s is the only expensive fp32 step, and s is constant over a channel.  With
+// s2 = s * 2^-30 and y = RN(1 / s2) (one IEEE reciprocal per channel), the sequence
+//     X0 = RN(w * y);  r = fma(-X0, s2, w);  X = fma(r, y, X0)
+// returns the correctly rounded quotient RN(w / s2) = RN(w / s) * 2^30 (Markstein's theorem: y
+// is a correctly rounded reciprocal, X0 is within one ulp, r is exact).  It needs s2 and y to be
+// normal numbers; the caller takes this path only for 2^-60 <= s <= 2^60.  The quotient comes
+// out already scaled to the fixed-point unit, so
+//     t  = X + kMagic     rounds X to a multiple of 2^30, ties to even (ulp of t is 2^30)
+//     qX = t - kMagic     = code * 2^30, exactly
+//     P  = cvt.rni(qX - X)   the perturbation in 2^-30 units (the difference is exact)
+// and the low byte of t's bit pattern is code + 128.
+constexpr float kMagic = 0x1.8001p53f;   // 1.5 * 2^53 + 128 * 2^30; mantissa field 0x400080
 
-    // ---- stage the channel in shared memory, absmax on the way
+__device__ __forceinline__ float div_scaled(float w, float y, float s2)
+{
+    const float x0 = __fmul_rn(w, y);
+    const float r = __fmaf_rn(-x0, s2, w);
+    return __fmaf_rn(r, y, x0);
+}
+
+__device__ __forceinline__ void squant_e_fast(float w, float y, float s2, unsigned &tbits, int &P)
+{
+    const float X = div_scaled(w, y, s2);
+    const float t = __fadd_rn(X, kMagic);
+    const float qX = __fsub_rn(t, kMagic);
+    P = __float2int_rn(__fsub_rn(qX, X));
+    tbits = __float_as_uint(t);
+}
+
+// Exact SQuant-K + Algorithm 3 on one 3x3 kernel from its weights in shared memory; codes are
+// written as biased bytes (code + 128).  Used for the few kernels the fast selection hands back.
+__device__ __forceinline__ void kernel9_exact(const float *wk, float y, float s2, unsigned char *cb,
+                                              int &e_out, int &v_out, int &idx_out)
+{
+    int P[9], q[9];
+    long long e = 0;
+#pragma unroll
+    for (int i = 0; i < 9; ++i) {
+        unsigned tb;
+        squant_e_fast(wk[i], y, s2, tb, P[i]);
+        q[i] = static_cast<int>(tb & 255u);
+        e += P[i];
+    }
+    int v = 0, idx = 0;
+    if (e != 0) {
+        const int sgn = e > 0 ? 1 : -1;
+        const long long abs_e = e > 0 ? e : -e;
+        const int k = flip_count(abs_e);
+        int flips = 0, last = -1, cand = -1;
+        for (int r = 0; r <= k; ++r) {
+            int best = 0, bi = -1;
+#pragma unroll
+            for (int i = 0; i < 9; ++i) {
+                const int key = sgn * P[i];
+                if (key > best) { best = key; bi = i; }
+            }
+            if (bi < 0) break;
+            if (r < k) {
+#pragma unroll
+                for (int i = 0; i < 9; ++i)
+                    if (i == bi) { P[i] -= sgn * kOne; q[i] -= sgn; }
+                last = bi;
+                ++flips;
+            } else {
+                cand = bi;
+            }
+        }
+        e -= static_cast<long long>(sgn) * flips * kOne;
+        const int pick = (static_cast<long long>(flips) * kOne > abs_e) ? last : cand;
+        if (pick >= 0) {
+            idx = pick;
+#pragma unroll
+            for (int i = 0; i < 9; ++i)
+                if (i == pick) v = P[i];
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < 9; ++i) cb[i] = static_cast<unsigned char>(q[i]);
+    e_out = static_cast<int>(e);
+    v_out = v;
+    idx_out = idx;
+}
+
+// Fast SQuant-K + Algorithm 3 on one 3x3 kernel whose perturbations P[0..8] are in registers and
+// whose biased code bytes are already staged at cb.
+//
+// Keys are the sign-normalised perturbations with the element index folded into their low four
+// bits ((key & ~15) | (15 - i)), so that the three largest can be tracked by value alone and
+// carry their positions.  This orders elements by (|P| >> 4, index); it equals Algorithm 2's
+// order (|P|, index) whenever the truncated values of neighbouring ranks differ, which is
+// checked.  Handled here: k = 0, k = 1, and k = 2 when it is Over SQuant - all but a few per
+// cent of random kernels.  Anything else (k = 2 Under, k >= 3, truncated values that tie or
+// are zero) returns false and the caller redoes the kernel with kernel9_exact.
+__device__ __forceinline__ bool kernel9_fast(const int (&P)[9], const float *wk, float y, float s2,
+                                             unsigned char *cb, int &e_out, int &v_out, int &idx_out)
+{
+    const int a = P[0] + P[1] + P[2], b = P[3] + P[4] + P[5], c = P[6] + P[7] + P[8];
+    const long long e = static_cast<long long>(a) + b + c;
+    e_out = 0;
+    v_out = 0;
+    idx_out = 0;
+    if (e == 0) return true;   // no flips, no candidate
+    const int sgn = e > 0 ? 1 : -1;
+    const long long abs_e = e > 0 ? e : -e;
+    const int k = flip_count(abs_e);
+    int m1 = 0, m2 = 0, m3 = 0;
+#pragma unroll
+    for (int i = 0; i < 9; ++i) {
+        const int key = ((P[i] * sgn) & ~15) | (15 - i);
+        const int t = min(m1, key);
+        m1 = max(m1, key);
+        const int u = min(m2, t);
+        m2 = max(m2, t);
+        m3 = max(m3, u);
+    }
+    const int c1 = m1 >> 4, c2 = m2 >> 4, c3 = m3 >> 4;
+    const bool over = (static_cast<long long>(k) << 30) > abs_e;
+    const bool ok = (k == 0) ? (c1 > c2) : (k <= 2 && (k == 1 || over) && c1 > c2 && c2 > c3);
+    if (!ok) return false;
+    if (k >= 1) {
+        const int i1 = 15 - (m1 & 15);
+        cb[i1] = static_cast<unsigned char>(cb[i1] - sgn);
+    }
+    if (k >= 2) {
+        const int i2 = 15 - (m2 & 15);
+        cb[i2] = static_cast<unsigned char>(cb[i2] - sgn);
+    }
+    // candidate: Over -> the k-th (last flipped), Under -> the (k+1)-th
+    const int mc = (k == 0 || (k == 1 && over)) ? m1 : m2;
+    const int idx = 15 - (mc & 15);
+    unsigned tb;
+    int Pc;
+    squant_e_fast(wk[idx], y, s2, tb, Pc);   // exact value of the candidate's perturbation
+    e_out = static_cast<int>(e - static_cast<long long>(sgn * k) * kOne);
+    v_out = over ? Pc - sgn * kOne : Pc;
+    idx_out = idx;
+    return true;
+}
+
+// ---------------------------------------------------------------- one output channel
+// Stages output channel m in the group's shared-memory slice (128-bit streaming loads when the
+// channel starts on a 16-byte boundary), takes its absmax on the way and returns the scale.
+// Ends with a group barrier, so the staged weights are visible to the whole group.
+__device__ __forceinline__ float stage_channel(const LayerDesc &L, int m, const Group &G,
+                                               unsigned char *slice, int qmax)
+{
+    const int NK = L.NK;
+    float *wbuf = reinterpret_cast<float *>(slice);
+    unsigned char *red = slice + L.off_red;
     const float *wg = L.w + static_cast<size_t>(m) * NK;
     float amax = 0.0f;
     if ((reinterpret_cast<uintptr_t>(wg) & 15) == 0) {
@@ -338,8 +471,51 @@ __device__ __forceinline__ void quantize_channel(const LayerDesc &L, int m, cons
             amax = fmaxf(amax, fabsf(t));
         }
     }
-    amax = group_absmax(G, amax, red);   // also makes wbuf visible to the whole group
-    const float s = (amax < 0x1p-100f) ? 1.0f : __fdiv_rn(amax, static_cast<float>(qmax));
+    amax = group_absmax(G, amax, red);
+    return (amax < 0x1p-100f) ? 1.0f : __fdiv_rn(amax, static_cast<float>(qmax));
+}
+
+// SQuant-C on the staged channel: channel sum, flip count, threshold of the radix select.
+struct ChannelStep {
+    long long ec;            // channel error sum after SQuant-C
+    int sgn_c, k_eff;        // direction and number of kernels to flip (k_eff = 0: none)
+    unsigned long long T;    // kernels whose candidate key is >= T are flipped
+};
+
+__device__ __forceinline__ ChannelStep channel_step(const LayerDesc &L, const Group &G,
+                                                    unsigned char *slice, long long esum,
+                                                    unsigned mode)
+{
+    int *vv = reinterpret_cast<int *>(slice + L.off_vv);
+    int *hist = reinterpret_cast<int *>(slice + L.off_hist);
+    unsigned char *red = slice + L.off_red;
+    int *bc = reinterpret_cast<int *>(red + 128);
+    ChannelStep c;
+    c.ec = 0; c.sgn_c = 0; c.k_eff = 0; c.T = ~0ull;
+    if ((mode & 4u) || L.cerr) c.ec = group_sum(G, esum, red);   // barrier: per-kernel data visible
+    else G.sync();
+    if ((mode & 4u) && c.ec != 0) {
+        c.sgn_c = c.ec > 0 ? 1 : -1;
+        const long long abs_e = c.ec > 0 ? c.ec : -c.ec;
+        const int kc = flip_count(abs_e);
+        if (kc > 0) c.k_eff = select_threshold(G, vv, L.N, c.sgn_c, kc, hist, bc, c.T);
+        c.ec -= static_cast<long long>(c.sgn_c) * c.k_eff * kOne;
+    }
+    return c;
+}
+
+// ---------------------------------------------------------------- channel body, any kernel size
+template <int KT>
+__device__ __forceinline__ void channel_body(const LayerDesc &L, int m, const Group &G,
+                                             unsigned char *slice, float s, unsigned mode)
+{
+    const int K = KT ? KT : L.K;
+    const int N = L.N, NK = L.NK;
+    float *wbuf = reinterpret_cast<float *>(slice);
+    int8_t *cbuf = reinterpret_cast<int8_t *>(slice + L.off_codes);
+    int *ev = reinterpret_cast<int *>(slice + L.off_ev);
+    int *vv = reinterpret_cast<int *>(slice + L.off_vv);
+    unsigned short *vi = reinterpret_cast<unsigned short *>(slice + L.off_vi);
 
     // ---- SQuant-E, SQuant-K, candidate: one thread per kernel
     // Without SQuant-K a kernel sum can reach K/2 and no longer fits 32 bits; it is then
@@ -372,18 +548,10 @@ __device__ __forceinline__ void quantize_channel(const LayerDesc &L, int m, cons
     }
 
     // ---- SQuant-C: Algorithm 2 on the channel, keys = the kernels' candidates
-    long long ec = 0;
-    int sgn_c = 0, k_eff = 0;
-    unsigned long long T = ~0ull;
-    if ((mode & 4u) || L.cerr) ec = group_sum(G, esum, red);   // sync: ev / vv / cbuf visible
-    else G.sync();
-    if ((mode & 4u) && ec != 0) {
-        sgn_c = ec > 0 ? 1 : -1;
-        const long long abs_e = ec > 0 ? ec : -ec;
-        const int kc = flip_count(abs_e);
-        if (kc > 0) k_eff = select_threshold(G, vv, N, sgn_c, kc, hist, bc, T);
-        ec -= static_cast<long long>(sgn_c) * k_eff * kOne;
-    }
+    const ChannelStep cs = channel_step(L, G, slice, esum, mode);
+    const long long ec = cs.ec;
+    const int sgn_c = cs.sgn_c, k_eff = cs.k_eff;
+    const unsigned long long T = cs.T;
 
     // ---- apply the channel flips, emit the kernels' error sums
     if (keep && (k_eff > 0 || kerr)) {
@@ -419,8 +587,279 @@ __device__ __forceinline__ void quantize_channel(const LayerDesc &L, int m, cons
     }
 }
 
+// ---------------------------------------------------------------- channel body, 3x3 fast path
+// Needs K = 9, N a multiple of 4, SQuant-K in the mode mask and 2^-60 <= s <= 2^60.
+// A thread owns four consecutive kernels = 36 consecutive weights: nine conflict-free 128-bit
+// shared loads in, nine conflict-free 32-bit stores of packed code bytes out.  Codes are staged
+// biased (code + 128) so that a flip is a plain byte +-1; the bias comes off in the copy-out.
+//
+// SQuant-C here needs ONE histogram, filled while the kernels are processed: bin = |v| >> 22 of
+// each kernel's candidate, positive and negative candidates counted in the two halves of one
+// 32-bit word.  Once the channel sum (hence the sign and k_c) is known, a warp scans the
+// histogram of that sign for the boundary bin; kernels above it are flipped, the few inside it
+// are collected in a list and ranked exactly (|v| descending, kernel index ascending).  A boundary
+// bin too crowded for the list (massive ties) falls back to the general radix select.
+constexpr int kListCap = 256;
+
+__device__ __forceinline__ void hist_add(int *hist, int v)
+{
+    if (v != 0) {
+        const int a = v > 0 ? v : -v;
+        atomicAdd(&hist[hist_slot(a >> 22)], v > 0 ? 1 : 0x10000);
+    }
+}
+
+__device__ __forceinline__ void channel_body_k9_fast(const LayerDesc &L, int m, const Group &G,
+                                                     unsigned char *slice, float s, unsigned mode)
+{
+    const int N = L.N, NK = L.NK;
+    const float *wbuf = reinterpret_cast<const float *>(slice);
+    unsigned char *cbuf = slice + L.off_codes;
+    int *ev = reinterpret_cast<int *>(slice + L.off_ev);
+    int *vv = reinterpret_cast<int *>(slice + L.off_vv);
+    unsigned char *vi = slice + L.off_vi;                       // N index bytes, then the redo list
+    unsigned short *redo = reinterpret_cast<unsigned short *>(vi + N);
+    const int redo_cap = N >> 1;
+    int *hist = reinterpret_cast<int *>(slice + L.off_hist);
+    unsigned char *red = slice + L.off_red;
+    int *bc = reinterpret_cast<int *>(red + 128);               // [0..3] scan result, [4] redo count, [5] list count
+    int2 *blist = reinterpret_cast<int2 *>(slice);              // boundary list: reuses the weights' space
+
+    for (int i = G.t; i < kHistBins; i += G.g) hist[i] = 0;
+    if (G.t == 0) { bc[4] = 0; bc[5] = 0; }
+    G.sync();
+
+    const float s2 = __fmul_rn(s, 0x1p-30f);
+    const float y = __frcp_rn(s2);
+    const int quads = N >> 2;
+    long long esum = 0;
+    for (int Q = G.t; Q < quads; Q += G.g) {
+        const float4 *src = reinterpret_cast<const float4 *>(wbuf) + Q * 9;
+        unsigned *dst = reinterpret_cast<unsigned *>(cbuf) + Q * 9;
+        float w[36];
+#pragma unroll
+        for (int j = 0; j < 9; ++j) {
+            const float4 t = src[j];
+            w[4 * j] = t.x; w[4 * j + 1] = t.y; w[4 * j + 2] = t.z; w[4 * j + 3] = t.w;
+        }
+        int P[36];
+#pragma unroll
+        for (int j = 0; j < 9; ++j) {
+            unsigned t0, t1, t2, t3;
+            squant_e_fast(w[4 * j], y, s2, t0, P[4 * j]);
+            squant_e_fast(w[4 * j + 1], y, s2, t1, P[4 * j + 1]);
+            squant_e_fast(w[4 * j + 2], y, s2, t2, P[4 * j + 2]);
+            squant_e_fast(w[4 * j + 3], y, s2, t3, P[4 * j + 3]);
+            dst[j] = __byte_perm(__byte_perm(t0, t1, 0x0040), __byte_perm(t2, t3, 0x0040), 0x5410);
+        }
+        int e4[4], v4[4];
+        unsigned i4 = 0;
+#pragma unroll
+        for (int kq = 0; kq < 4; ++kq) {
+            int Pk[9];
+#pragma unroll
+            for (int i = 0; i < 9; ++i) Pk[i] = P[9 * kq + i];
+            const int n = 4 * Q + kq;
+            int idx;
+            if (!kernel9_fast(Pk, wbuf + n * 9, y, s2, cbuf + n * 9, e4[kq], v4[kq], idx)) {
+                const int pos = atomicAdd(&bc[4], 1);
+                if (pos < redo_cap) {
+                    redo[pos] = static_cast<unsigned short>(n);
+                    e4[kq] = 0;   // e, v, idx are filled in by the redo pass
+                    v4[kq] = 0;
+                    idx = 0;
+                } else {
+                    kernel9_exact(wbuf + n * 9, y, s2, cbuf + n * 9, e4[kq], v4[kq], idx);
+                }
+            }
+            hist_add(hist, v4[kq]);
+            i4 |= static_cast<unsigned>(idx) << (8 * kq);
+            esum += e4[kq];
+        }
+        reinterpret_cast<int4 *>(ev)[Q] = make_int4(e4[0], e4[1], e4[2], e4[3]);
+        reinterpret_cast<int4 *>(vv)[Q] = make_int4(v4[0], v4[1], v4[2], v4[3]);
+        reinterpret_cast<unsigned *>(vi)[Q] = i4;
+    }
+    G.sync();
+    {   // kernels handed back by the fast selection, redone exactly, densely over the group
+        const int nredo = min(bc[4], redo_cap);
+        for (int i = G.t; i < nredo; i += G.g) {
+            const int n = redo[i];
+            int e1, v, idx;
+            kernel9_exact(wbuf + n * 9, y, s2, cbuf + n * 9, e1, v, idx);
+            ev[n] = e1;
+            vv[n] = v;
+            vi[n] = static_cast<unsigned char>(idx);
+            hist_add(hist, v);
+            esum += e1;
+        }
+    }
+
+    // ---- SQuant-C: channel sum, boundary bin
+    long long ec = 0;
+    if ((mode & 4u) || L.cerr) ec = group_sum(G, esum, red);   // barrier: per-kernel data, histogram visible
+    else G.sync();
+    int sgn_c = 0, k_eff = 0;
+    int t_all = 0x7fffffff;     // candidates with v * sgn_c >= t_all are flipped outright
+    int t_list = 0x7fffffff;    // those in [t_list, t_all) go to the boundary list
+    int rem = 0, cb = 0;
+    unsigned long long T64 = ~0ull;
+    bool wide = false;          // fallback: compare 48-bit keys against T64
+    if ((mode & 4u) && ec != 0) {
+        sgn_c = ec > 0 ? 1 : -1;
+        const long long abs_e = ec > 0 ? ec : -ec;
+        const int kc = flip_count(abs_e);
+        if (kc > 0) {
+            if (G.t < 32) {
+                const int lane = G.t, grp = 31 - lane, sh = sgn_c > 0 ? 0 : 16;
+                int c[8], s8 = 0;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) { c[j] = (hist[(j << 5) | grp] >> sh) & 0xffff; s8 += c[j]; }
+                int incl = s8;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int t = __shfl_up_sync(kFull, incl, o);
+                    if (lane >= o) incl += t;
+                }
+                const int total = __shfl_sync(kFull, incl, 31);
+                const int want = min(kc, total);
+                const unsigned bal = __ballot_sync(kFull, incl >= want);
+                if (want <= 0) {
+                    if (lane == 0) { bc[0] = -1; bc[1] = 0; bc[2] = 0; bc[3] = 0; }
+                } else if (lane == __ffs(bal) - 1) {
+                    int cum = incl - s8, b = -1, cnt = 0;
+#pragma unroll
+                    for (int j = 7; j >= 0; --j) {
+                        if (b < 0) {
+                            if (cum + c[j] >= want) { b = grp * 8 + j; cnt = c[j]; }
+                            else cum += c[j];
+                        }
+                    }
+                    bc[0] = b; bc[1] = want - cum; bc[2] = cnt; bc[3] = want;
+                }
+            }
+            G.sync();
+            const int b = bc[0];
+            rem = bc[1];
+            cb = bc[2];
+            k_eff = bc[3];
+            if (b >= 0) {
+                if (cb == rem) {                 // whole boundary bin flipped
+                    t_all = max(b << 22, 1);   // 0 is "no candidate"
+                } else if (cb <= kListCap) {     // rank the boundary bin exactly
+                    t_all = (b + 1) << 22;       // b + 1 = 256 gives 2^30, above every |v|
+                    t_list = max(b << 22, 1);
+                } else {                         // crowded bin: general radix select on 48-bit keys
+                    wide = true;
+                    G.sync();                    // everyone has read bc before the select reuses it
+                    k_eff = select_threshold(G, vv, N, sgn_c, kc, hist, bc, T64);
+                }
+            } else {
+                k_eff = 0;
+            }
+            ec -= static_cast<long long>(sgn_c) * k_eff * kOne;
+        }
+    }
+
+    // ---- apply the channel flips, emit the kernels' error sums (four kernels per thread)
+    float *kerr = L.kerr ? L.kerr + static_cast<size_t>(m) * N : nullptr;
+    const bool listing = t_list != 0x7fffffff;
+    if (k_eff > 0 || kerr) {
+        const bool vec = kerr && !listing && (reinterpret_cast<uintptr_t>(kerr) & 15) == 0;
+        for (int Q = G.t; Q < quads; Q += G.g) {
+            const int4 e4 = reinterpret_cast<const int4 *>(ev)[Q];
+            int e[4] = {e4.x, e4.y, e4.z, e4.w};
+            bool listed[4] = {false, false, false, false};
+            if (k_eff > 0) {
+                const int4 v4 = reinterpret_cast<const int4 *>(vv)[Q];
+                const int v[4] = {v4.x, v4.y, v4.z, v4.w};
+                const unsigned i4 = reinterpret_cast<const unsigned *>(vi)[Q];
+#pragma unroll
+                for (int kq = 0; kq < 4; ++kq) {
+                    const int n = 4 * Q + kq;
+                    const int a = v[kq] * sgn_c;
+                    bool take;
+                    if (wide) {
+                        const unsigned long long ck = cand_key(v[kq], sgn_c, n);
+                        take = ck != 0 && ck >= T64;
+                    } else {
+                        take = a >= t_all;
+                        if (!take && a >= t_list) {
+                            listed[kq] = true;
+                            const int pos = atomicAdd(&bc[5], 1);
+                            if (pos < kListCap) blist[pos] = make_int2(a, n);
+                        }
+                    }
+                    if (take) {
+                        e[kq] -= sgn_c * kOne;
+                        unsigned char *bp = cbuf + n * 9 + ((i4 >> (8 * kq)) & 255u);
+                        *bp = static_cast<unsigned char>(*bp - sgn_c);
+                    }
+                }
+            }
+            if (kerr) {
+                float4 f;
+                f.x = __fmul_rn(__int2float_rn(e[0]), 0x1p-30f);
+                f.y = __fmul_rn(__int2float_rn(e[1]), 0x1p-30f);
+                f.z = __fmul_rn(__int2float_rn(e[2]), 0x1p-30f);
+                f.w = __fmul_rn(__int2float_rn(e[3]), 0x1p-30f);
+                if (vec) {
+                    __stcs(reinterpret_cast<float4 *>(kerr) + Q, f);
+                } else {   // listed kernels are written by the ranking step below
+                    if (!listed[0]) kerr[4 * Q] = f.x;
+                    if (!listed[1]) kerr[4 * Q + 1] = f.y;
+                    if (!listed[2]) kerr[4 * Q + 2] = f.z;
+                    if (!listed[3]) kerr[4 * Q + 3] = f.w;
+                }
+            }
+        }
+    }
+    G.sync();
+    if (listing) {   // exact rank inside the boundary bin: cb entries, the first `rem` are flipped
+        for (int i = G.t; i < cb; i += G.g) {
+            const int2 me = blist[i];
+            int rank = 0;
+            for (int j = 0; j < cb; ++j) {
+                const int2 o = blist[j];
+                rank += (o.x > me.x || (o.x == me.x && o.y < me.y)) ? 1 : 0;
+            }
+            int e1 = ev[me.y];
+            if (rank < rem) {
+                e1 -= sgn_c * kOne;
+                unsigned char *bp = cbuf + me.y * 9 + vi[me.y];
+                *bp = static_cast<unsigned char>(*bp - sgn_c);
+            }
+            if (kerr) kerr[me.y] = __fmul_rn(__int2float_rn(e1), 0x1p-30f);
+        }
+        G.sync();
+    }
+
+    // ---- codes (bias removed), scale, channel error
+    int8_t *cg = L.codes + static_cast<size_t>(m) * NK;
+    if ((reinterpret_cast<uintptr_t>(cg) & 15) == 0) {
+        const int nv = NK >> 4;
+        const int4 *src = reinterpret_cast<const int4 *>(cbuf);
+        int4 *dst = reinterpret_cast<int4 *>(cg);
+        for (int i = G.t; i < nv; i += G.g) {
+            int4 t = src[i];
+            t.x ^= 0x80808080; t.y ^= 0x80808080; t.z ^= 0x80808080; t.w ^= 0x80808080;
+            __stcs(dst + i, t);
+        }
+        for (int i = (nv << 4) + G.t; i < NK; i += G.g) cg[i] = static_cast<int8_t>(cbuf[i] ^ 0x80);
+    } else {
+        for (int i = G.t; i < NK; i += G.g) cg[i] = static_cast<int8_t>(cbuf[i] ^ 0x80);
+    }
+    if (G.t == 0) {
+        L.scales[m] = s;
+        if (L.cerr) L.cerr[m] = __fmul_rn(__ll2float_rn(ec), 0x1p-30f);
+    }
+}
+
 // ---------------------------------------------------------------- grouped launch
-__global__ void __launch_bounds__(kCtaThreads)
+#ifndef SQ_MIN_CTAS
+#define SQ_MIN_CTAS 2
+#endif
+__global__ void __launch_bounds__(kCtaThreads, SQ_MIN_CTAS)
 squant_model_kernel(const LayerDesc *__restrict__ layers, const Item *__restrict__ items, int qmax,
                     unsigned mode)
 {
@@ -435,9 +874,17 @@ squant_model_kernel(const LayerDesc *__restrict__ layers, const Item *__restrict
     const int m = it.ch0 + gi;
     if (m >= L.M) return;   // the whole group leaves together; it shares no barrier with others
     unsigned char *slice = smem + static_cast<size_t>(gi) * L.slice_bytes;
-    if (L.K == 1) quantize_channel<1>(L, m, G, slice, qmax, mode);
-    else if (L.K == 9) quantize_channel<9>(L, m, G, slice, qmax, mode);
-    else quantize_channel<0>(L, m, G, slice, qmax, mode);
+    const float s = stage_channel(L, m, G, slice, qmax);
+    if (L.K == 1) {
+        channel_body<1>(L, m, G, slice, s, mode);
+    } else if (L.K == 9) {
+        if ((L.N & 3) == 0 && (mode & 2u) && s >= 0x1p-60f && s <= 0x1p60f)
+            channel_body_k9_fast(L, m, G, slice, s, mode);
+        else
+            channel_body<9>(L, m, G, slice, s, mode);
+    } else {
+        channel_body<0>(L, m, G, slice, s, mode);
+    }
 }
 
 }  // namespace sq
