@@ -62,6 +62,8 @@ extern "C" {
 #define SQUANT_ERR_TOO_WIDE (-6)    /* one output channel does not fit the on-chip path */
 #define SQUANT_ERR_CUDA (-7)        /* a CUDA runtime call failed; see squant_last_cuda_error() */
 #define SQUANT_ERR_NOMEM (-8)       /* host or device allocation failed */
+#define SQUANT_ERR_TIMEOUT (-10)    /* a kernel gave up a bounded wait on an asynchronous copy; the
+                                       outputs of that launch are incomplete */
 #define SQUANT_ERR_LIMIT (-9)       /* the layer needs more launch-table entries than the fixed
                                        table of squant_quantize_layer_noalloc holds */
 
@@ -165,6 +167,15 @@ int squant_plan_info(const squant_layer *layers, int32_t n_layers, const squant_
 #define SQUANT_NOALLOC_TABLE_BYTES (256 + 8 * SQUANT_NOALLOC_MAX_CTAS)
 int squant_quantize_layer_noalloc(const squant_layer *layer, const squant_options *opt,
                                   void *cuda_stream);
+
+/*
+ * Waits for all work on the current device and reports whether any kernel of this library gave
+ * up one of its bounded waits since the last query (every wait inside the kernels - they only
+ * wait for their own asynchronous copies - has an iteration limit, after which the affected
+ * thread group records the fact, writes nothing and leaves).  Returns SQUANT_OK,
+ * SQUANT_ERR_TIMEOUT (and clears the record) or SQUANT_ERR_CUDA.
+ */
+int squant_device_status(void);
 
 /* Number of kernels this library has launched in this process (all entry points). */
 int64_t squant_launch_count(void);

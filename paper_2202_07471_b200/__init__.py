@@ -4,13 +4,13 @@
 The CUDA library is loaded on first use and there is no fallback when it is missing.
 """
 from .binding import (FLAG_NARROW_RANGE, NOALLOC_MAX_CTAS, MODE_C, MODE_E, MODE_EKC, MODE_K, LayerBuffers, ModelCall,
-                      SquantError, alloc_outputs, load_library, squant_launch_count,
+                      SquantError, alloc_outputs, load_library, squant_device_status, squant_launch_count,
                       squant_plan_info, squant_quantize_layer, squant_quantize_layer_noalloc,
                       squant_quantize_model,
                       squant_quantize_model_host, squant_shutdown)
 
 __all__ = ["FLAG_NARROW_RANGE", "NOALLOC_MAX_CTAS", "MODE_C", "MODE_E", "MODE_EKC", "MODE_K", "LayerBuffers",
-           "ModelCall", "SquantError", "alloc_outputs", "load_library", "squant_launch_count",
+           "ModelCall", "SquantError", "alloc_outputs", "load_library", "squant_device_status", "squant_launch_count",
            "squant_plan_info", "squant_quantize_layer", "squant_quantize_layer_noalloc",
            "squant_quantize_model",
            "squant_quantize_model_host", "squant_shutdown"]

@@ -22,7 +22,7 @@ LIB_PATH = os.path.join(_HERE, "libsquant.so")
 NOALLOC_MAX_CTAS = 32768
 
 EXPORTS = ("squant_quantize_layer", "squant_quantize_layer_noalloc", "squant_quantize_model", "squant_quantize_model_host",
-           "squant_plan_info", "squant_launch_count", "squant_strerror", "squant_last_cuda_error",
+           "squant_plan_info", "squant_device_status", "squant_launch_count", "squant_strerror", "squant_last_cuda_error",
            "squant_shutdown")
 
 
@@ -63,7 +63,7 @@ def load_library() -> ctypes.CDLL:
     lib.squant_quantize_model_host.argtypes = [lp, ctypes.c_int32, op, vp]
     lib.squant_plan_info.argtypes = [lp, ctypes.c_int32, op, i32p, i32p, i32p]
     for f in ("squant_quantize_layer", "squant_quantize_layer_noalloc", "squant_quantize_model", "squant_quantize_model_host",
-              "squant_plan_info", "squant_shutdown"):
+              "squant_plan_info", "squant_device_status", "squant_shutdown"):
         getattr(lib, f).restype = ctypes.c_int
     lib.squant_launch_count.restype = ctypes.c_int64
     lib.squant_strerror.restype = ctypes.c_char_p
@@ -209,6 +209,11 @@ def squant_plan_info(shapes: Sequence[Sequence[int]], bits: int = 4, mode: int =
     _check(load_library().squant_plan_info(arr, len(shapes), ctypes.byref(opt), ctypes.byref(g),
                                            ctypes.byref(t), ctypes.byref(s)))
     return {"grid_ctas": g.value, "cta_threads": t.value, "dynamic_smem_bytes": s.value}
+
+
+def squant_device_status() -> None:
+    """Synchronise the current device; raise SquantError(-10) if a kernel gave up a bounded wait."""
+    _check(load_library().squant_device_status())
 
 
 def squant_launch_count() -> int:

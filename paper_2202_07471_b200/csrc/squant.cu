@@ -409,6 +409,18 @@ int squant_plan_info(const squant_layer *layers, int32_t n_layers, const squant_
     return SQUANT_OK;
 }
 
+int squant_device_status(void)
+{
+    std::lock_guard<std::mutex> lock(g_mutex);
+    SQ_CUDA(cudaDeviceSynchronize());
+    int st = 0;
+    SQ_CUDA(cudaMemcpyFromSymbol(&st, sq::g_device_status, sizeof(int)));
+    if (st == 0) return SQUANT_OK;
+    const int zero = 0;
+    SQ_CUDA(cudaMemcpyToSymbol(sq::g_device_status, &zero, sizeof(int)));
+    return SQUANT_ERR_TIMEOUT;
+}
+
 int64_t squant_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 const char *squant_strerror(int code)
@@ -423,6 +435,7 @@ const char *squant_strerror(int code)
         case SQUANT_ERR_TOO_WIDE: return "an output channel (cin*kh*kw) does not fit the on-chip path";
         case SQUANT_ERR_CUDA: return "a CUDA runtime call failed (see squant_last_cuda_error)";
         case SQUANT_ERR_NOMEM: return "out of host or device memory";
+        case SQUANT_ERR_TIMEOUT: return "a kernel gave up a bounded wait on an asynchronous copy; outputs of that launch are incomplete";
         case SQUANT_ERR_LIMIT: return "the layer needs more thread blocks than the fixed launch table of squant_quantize_layer_noalloc holds (SQUANT_NOALLOC_MAX_CTAS); split it by output-channel range";
         default: return "unknown squant error code";
     }

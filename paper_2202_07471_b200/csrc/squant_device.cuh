@@ -53,6 +53,61 @@ struct Group {
     }
 };
 
+// ---------------------------------------------------------------- bulk async copies (TMA)
+// Set to a non-zero code by a kernel whose bounded wait on a bulk copy ran out; read and cleared
+// by squant_device_status().
+__device__ int g_device_status = 0;
+constexpr int kWaitIters = 1 << 22;   // each try_wait itself blocks for a hardware time slice
+
+__device__ __forceinline__ unsigned smem_addr(const void *p)
+{
+    return static_cast<unsigned>(__cvta_generic_to_shared(p));
+}
+
+__device__ __forceinline__ void mbar_init(void *bar, unsigned count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+
+// One-dimensional bulk copy global -> shared of `bytes` (multiple of 16, both sides 16-byte
+// aligned, no multicast), completion counted on `bar`.
+__device__ __forceinline__ void bulk_load(void *dst, const void *src, unsigned bytes, void *bar)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(smem_addr(dst)),
+                 "l"(src), "r"(bytes), "r"(smem_addr(bar))
+                 : "memory");
+}
+
+// Bounded wait for phase `parity` of `bar`.  False if the limit ran out.
+__device__ __forceinline__ bool mbar_wait(void *bar, unsigned parity)
+{
+    const unsigned a = smem_addr(bar);
+    for (int it = 0; it < kWaitIters; ++it) {
+        unsigned done;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(done) : "r"(a), "r"(parity) : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+
+// Bulk copy shared -> global of `bytes` (multiple of 16, both sides 16-byte aligned), issued by
+// one thread after the writers' barrier; the caller waits with bulk_store_wait before the shared
+// memory may be reused or the CTA exits.
+__device__ __forceinline__ void bulk_store(void *dst, const void *src, unsigned bytes)
+{
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(smem_addr(src)), "r"(bytes) : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+
+__device__ __forceinline__ void bulk_store_wait()
+{
+    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+}
+
 // ---------------------------------------------------------------- group-wide reductions
 // `red` points at 16 eight-byte slots owned by the group.
 __device__ __forceinline__ float group_absmax(const Group &G, float v, void *red)
@@ -309,8 +364,8 @@ __device__ __forceinline__ int select_threshold(const Group &G, const int *vv, i
 //     t  = X + kMagic     rounds X to a multiple of 2^30, ties to even (ulp of t is 2^30)
 //     qX = t - kMagic     = code * 2^30, exactly
 //     P  = cvt.rni(qX - X)   the perturbation in 2^-30 units (the difference is exact)
-// and the low byte of t's bit pattern is code + 128.
-constexpr float kMagic = 0x1.8001p53f;   // 1.5 * 2^53 + 128 * 2^30; mantissa field 0x400080
+// and the low byte of t's bit pattern is the code in two's complement.
+constexpr float kMagic = 0x1.8p53f;   // 1.5 * 2^53: mantissa field 0x400000, low byte 0
 
 __device__ __forceinline__ float div_scaled(float w, float y, float s2)
 {
@@ -319,17 +374,24 @@ __device__ __forceinline__ float div_scaled(float w, float y, float s2)
     return __fmaf_rn(r, y, x0);
 }
 
-__device__ __forceinline__ void squant_e_fast(float w, float y, float s2, unsigned &tbits, int &P)
+__device__ __forceinline__ void squant_e_fastf(float w, float y, float s2, unsigned &tbits, float &Pf)
 {
     const float X = div_scaled(w, y, s2);
     const float t = __fadd_rn(X, kMagic);
     const float qX = __fsub_rn(t, kMagic);
-    P = __float2int_rn(__fsub_rn(qX, X));
+    Pf = __fsub_rn(qX, X);   // exact; |Pf| <= 2^29 (+ one ulp of qmax * 2^30 for the absmax element)
     tbits = __float_as_uint(t);
 }
 
+__device__ __forceinline__ void squant_e_fast(float w, float y, float s2, unsigned &tbits, int &P)
+{
+    float Pf;
+    squant_e_fastf(w, y, s2, tbits, Pf);
+    P = __float2int_rn(Pf);
+}
+
 // Exact SQuant-K + Algorithm 3 on one 3x3 kernel from its weights in shared memory; codes are
-// written as biased bytes (code + 128).  Used for the few kernels the fast selection hands back.
+// written as bytes.  Used for the few kernels the fast selection hands back.
 __device__ __forceinline__ void kernel9_exact(const float *wk, float y, float s2, unsigned char *cb,
                                               int &e_out, int &v_out, int &idx_out)
 {
@@ -382,65 +444,81 @@ __device__ __forceinline__ void kernel9_exact(const float *wk, float y, float s2
     idx_out = idx;
 }
 
-// Fast SQuant-K + Algorithm 3 on one 3x3 kernel whose perturbations P[0..8] are in registers and
-// whose biased code bytes are already staged at cb.
+// Fast SQuant-K + Algorithm 3 on one 3x3 kernel whose exact perturbations Pf[0..8] (floats, in
+// 2^-30 units, before the conversion to integers) are in registers and whose code bytes
+// are already staged at cb.  Straight-line on purpose: every lane runs the same instructions and
+// the rare hand-back to kernel9_exact is a returned flag.
 //
-// Keys are the sign-normalised perturbations with the element index folded into their low four
-// bits ((key & ~15) | (15 - i)), so that the three largest can be tracked by value alone and
-// carry their positions.  This orders elements by (|P| >> 4, index); it equals Algorithm 2's
-// order (|P|, index) whenever the truncated values of neighbouring ranks differ, which is
-// checked.  Handled here: k = 0, k = 1, and k = 2 when it is Over SQuant - all but a few per
-// cent of random kernels.  Anything else (k = 2 Under, k >= 3, truncated values that tie or
-// are zero) returns false and the caller redoes the kernel with kernel9_exact.
-__device__ __forceinline__ bool kernel9_fast(const int (&P)[9], const float *wk, float y, float s2,
+// Sign, flip count and Over/Under come from a float sum of the perturbations.  That sum is
+// within 4096 units of the exact integer sum e (nine conversions round by <= 0.5 each, eight
+// additions by <= 256 each), and every decision boundary - 0, (j - 1/2) * 2^30 for k, j * 2^30 for
+// Over - is a multiple of 2^29; so with v = |sum| / 2^29 the decisions are exact whenever v is at
+// least 2^-17 away from an integer, and j = floor(v) gives k = (j + 1) / 2 and Over = (j odd).
+// Closer than that the kernel is handed back (an exactly zero integer sum is recognised first).
+// The exact |e| is still summed in integers (mod 2^32) for the error sum that is emitted.
+//
+// Selection: keys are the sign-normalised integer perturbations with the element index folded
+// into their low four bits, (P & ~15) | (15 - i), so the three largest can be tracked by value
+// alone and carry their positions.  This orders by (P >> 4, index); it equals Algorithm 2's
+// order (P, index) whenever the truncated values of neighbouring ranks differ, which is checked.
+// Handled: j = 0 (k = 0), j = 1 (k = 1, Over), j = 2 (k = 1, Under), j = 3 (k = 2, Over).
+__device__ __forceinline__ bool kernel9_fast(const float (&Pf)[9], const float *wk, float y, float s2,
                                              unsigned char *cb, int &e_out, int &v_out, int &idx_out)
 {
-    const int a = P[0] + P[1] + P[2], b = P[3] + P[4] + P[5], c = P[6] + P[7] + P[8];
-    const long long e = static_cast<long long>(a) + b + c;
-    e_out = 0;
-    v_out = 0;
-    idx_out = 0;
-    if (e == 0) return true;   // no flips, no candidate
-    const int sgn = e > 0 ? 1 : -1;
-    const long long abs_e = e > 0 ? e : -e;
-    const int k = flip_count(abs_e);
+    const float ef = __fadd_rn(__fadd_rn(__fadd_rn(__fadd_rn(Pf[0], Pf[1]), __fadd_rn(Pf[2], Pf[3])),
+                                         __fadd_rn(__fadd_rn(Pf[4], Pf[5]), __fadd_rn(Pf[6], Pf[7]))),
+                               Pf[8]);
+    const float sgn_f = copysignf(1.0f, ef);
+    const int sgn = ef < 0.0f ? -1 : 1;
+    const float v = __fmul_rn(fabsf(ef), 0x1p-29f);
+    const bool near = fabsf(__fsub_rn(v, rintf(v))) < 0x1p-17f;
+    const int j = __float2int_rd(v);
     int m1 = 0, m2 = 0, m3 = 0;
+    unsigned eabs = 0;   // |e| mod 2^32
 #pragma unroll
     for (int i = 0; i < 9; ++i) {
-        const int key = ((P[i] * sgn) & ~15) | (15 - i);
+        const int Ps = __float2int_rn(__fmul_rn(Pf[i], sgn_f));
+        eabs += static_cast<unsigned>(Ps);
+        const int key = (Ps & ~15) | (15 - i);
         const int t = min(m1, key);
         m1 = max(m1, key);
         const int u = min(m2, t);
         m2 = max(m2, t);
         m3 = max(m3, u);
     }
-    const int c1 = m1 >> 4, c2 = m2 >> 4, c3 = m3 >> 4;
-    const bool over = (static_cast<long long>(k) << 30) > abs_e;
-    const bool ok = (k == 0) ? (c1 > c2) : (k <= 2 && (k == 1 || over) && c1 > c2 && c2 > c3);
-    if (!ok) return false;
-    if (k >= 1) {
+    const bool d12 = (m1 >> 4) > (m2 >> 4), d23 = (m2 >> 4) > (m3 >> 4);
+    const bool zero = near & (j == 0) & (eabs == 0u);   // e == 0: no flips, no candidate
+    const bool ok = zero | (!near & d12 & ((j <= 1) | (d23 & (j <= 3))));
+    // ok with j >= 1 implies m1 >= 16, ok with j >= 2 implies m2 >= 16: the indices below are 0..8
+    if (ok & (j >= 1)) {
         const int i1 = 15 - (m1 & 15);
         cb[i1] = static_cast<unsigned char>(cb[i1] - sgn);
     }
-    if (k >= 2) {
+    if (ok & (j == 3)) {
         const int i2 = 15 - (m2 & 15);
         cb[i2] = static_cast<unsigned char>(cb[i2] - sgn);
     }
-    // candidate: Over -> the k-th (last flipped), Under -> the (k+1)-th
-    const int mc = (k == 0 || (k == 1 && over)) ? m1 : m2;
-    const int idx = 15 - (mc & 15);
+    // candidate: Over (j odd) -> the k-th (last flipped), Under -> the (k+1)-th
+    const int mc = (j <= 1) ? m1 : m2;
+    const int idx = 15 - (mc & 15);   // at most 15: stays inside the staged channel
     unsigned tb;
-    int Pc;
-    squant_e_fast(wk[idx], y, s2, tb, Pc);   // exact value of the candidate's perturbation
-    e_out = static_cast<int>(e - static_cast<long long>(sgn * k) * kOne);
-    v_out = over ? Pc - sgn * kOne : Pc;
+    float Pcf;
+    squant_e_fastf(wk[idx], y, s2, tb, Pcf);   // exact value of the candidate's perturbation
+    const int Pc = __float2int_rn(__fmul_rn(Pcf, sgn_f));
+    const int vs = (j & 1) ? Pc - kOne : Pc;
+    const unsigned k = static_cast<unsigned>(j + 1) >> 1;
+    e_out = sgn * static_cast<int>(eabs - (k << 30));
+    v_out = zero ? 0 : sgn * vs;
     idx_out = idx;
-    return true;
+    return !ok;
 }
 
 // ---------------------------------------------------------------- one output channel
-// Stages output channel m in the group's shared-memory slice (128-bit streaming loads when the
-// channel starts on a 16-byte boundary), takes its absmax on the way and returns the scale.
+// Stages output channel m in the group's shared-memory slice, takes its absmax and returns the
+// scale (0 if the staging wait ran out: the caller must leave without writing).  A channel that
+// starts on a 16-byte boundary and whose length is a multiple of four floats arrives by ONE bulk
+// asynchronous copy issued by the group's first thread (the whole channel is in flight at once,
+// no registers or load instructions spent on it); anything else is fetched with plain loads.
 // Ends with a group barrier, so the staged weights are visible to the whole group.
 __device__ __forceinline__ float stage_channel(const LayerDesc &L, int m, const Group &G,
                                                unsigned char *slice, int qmax)
@@ -448,21 +526,28 @@ __device__ __forceinline__ float stage_channel(const LayerDesc &L, int m, const 
     const int NK = L.NK;
     float *wbuf = reinterpret_cast<float *>(slice);
     unsigned char *red = slice + L.off_red;
+    unsigned long long *bar = reinterpret_cast<unsigned long long *>(red + 192);
+    int *flag = reinterpret_cast<int *>(red + 200);
     const float *wg = L.w + static_cast<size_t>(m) * NK;
     float amax = 0.0f;
-    if ((reinterpret_cast<uintptr_t>(wg) & 15) == 0) {
+    if ((reinterpret_cast<uintptr_t>(wg) & 15) == 0 && (NK & 3) == 0) {
+        if (G.t == 0) {
+            *flag = 0;
+            mbar_init(bar, 1);
+            bulk_load(wbuf, wg, static_cast<unsigned>(NK) * 4u, bar);
+        }
+        G.sync();   // barrier initialised before anyone polls it
+        if (!mbar_wait(bar, 0)) *flag = 1;
         const int nv = NK >> 2;
-        const float4 *src = reinterpret_cast<const float4 *>(wg);
-        float4 *dst = reinterpret_cast<float4 *>(wbuf);
+        const float4 *src = reinterpret_cast<const float4 *>(wbuf);
         for (int i = G.t; i < nv; i += G.g) {
-            const float4 t = __ldcs(src + i);
-            dst[i] = t;
+            const float4 t = src[i];
             amax = fmaxf(fmaxf(amax, fabsf(t.x)), fmaxf(fabsf(t.y), fmaxf(fabsf(t.z), fabsf(t.w))));
         }
-        for (int i = (nv << 2) + G.t; i < NK; i += G.g) {
-            const float t = __ldcs(wg + i);
-            wbuf[i] = t;
-            amax = fmaxf(amax, fabsf(t));
+        amax = group_absmax(G, amax, red);
+        if (*flag) {   // group-uniform after the barrier inside group_absmax
+            if (G.t == 0) atomicExch(&g_device_status, 1);
+            return 0.0f;
         }
     } else {
         for (int i = G.t; i < NK; i += G.g) {
@@ -470,8 +555,8 @@ __device__ __forceinline__ float stage_channel(const LayerDesc &L, int m, const 
             wbuf[i] = t;
             amax = fmaxf(amax, fabsf(t));
         }
+        amax = group_absmax(G, amax, red);
     }
-    amax = group_absmax(G, amax, red);
     return (amax < 0x1p-100f) ? 1.0f : __fdiv_rn(amax, static_cast<float>(qmax));
 }
 
@@ -590,8 +675,8 @@ __device__ __forceinline__ void channel_body(const LayerDesc &L, int m, const Gr
 // ---------------------------------------------------------------- channel body, 3x3 fast path
 // Needs K = 9, N a multiple of 4, SQuant-K in the mode mask and 2^-60 <= s <= 2^60.
 // A thread owns four consecutive kernels = 36 consecutive weights: nine conflict-free 128-bit
-// shared loads in, nine conflict-free 32-bit stores of packed code bytes out.  Codes are staged
-// biased (code + 128) so that a flip is a plain byte +-1; the bias comes off in the copy-out.
+// shared loads in, nine conflict-free 32-bit stores of packed code bytes out; flips are byte
+// read-modify-writes on the staged codes.
 //
 // SQuant-C here needs ONE histogram, filled while the kernels are processed: bin = |v| >> 22 of
 // each kernel's candidate, positive and negative candidates counted in the two halves of one
@@ -642,35 +727,33 @@ __device__ __forceinline__ void channel_body_k9_fast(const LayerDesc &L, int m, 
             const float4 t = src[j];
             w[4 * j] = t.x; w[4 * j + 1] = t.y; w[4 * j + 2] = t.z; w[4 * j + 3] = t.w;
         }
-        int P[36];
+        float P[36];
 #pragma unroll
         for (int j = 0; j < 9; ++j) {
             unsigned t0, t1, t2, t3;
-            squant_e_fast(w[4 * j], y, s2, t0, P[4 * j]);
-            squant_e_fast(w[4 * j + 1], y, s2, t1, P[4 * j + 1]);
-            squant_e_fast(w[4 * j + 2], y, s2, t2, P[4 * j + 2]);
-            squant_e_fast(w[4 * j + 3], y, s2, t3, P[4 * j + 3]);
+            squant_e_fastf(w[4 * j], y, s2, t0, P[4 * j]);
+            squant_e_fastf(w[4 * j + 1], y, s2, t1, P[4 * j + 1]);
+            squant_e_fastf(w[4 * j + 2], y, s2, t2, P[4 * j + 2]);
+            squant_e_fastf(w[4 * j + 3], y, s2, t3, P[4 * j + 3]);
             dst[j] = __byte_perm(__byte_perm(t0, t1, 0x0040), __byte_perm(t2, t3, 0x0040), 0x5410);
         }
         int e4[4], v4[4];
-        unsigned i4 = 0;
+        unsigned i4 = 0, overflow = 0;
 #pragma unroll
         for (int kq = 0; kq < 4; ++kq) {
-            int Pk[9];
+            float Pk[9];
 #pragma unroll
             for (int i = 0; i < 9; ++i) Pk[i] = P[9 * kq + i];
             const int n = 4 * Q + kq;
             int idx;
-            if (!kernel9_fast(Pk, wbuf + n * 9, y, s2, cbuf + n * 9, e4[kq], v4[kq], idx)) {
+            const bool again = kernel9_fast(Pk, wbuf + n * 9, y, s2, cbuf + n * 9, e4[kq], v4[kq], idx);
+            if (again) {   // e, v, idx are filled in by the redo pass
                 const int pos = atomicAdd(&bc[4], 1);
-                if (pos < redo_cap) {
-                    redo[pos] = static_cast<unsigned short>(n);
-                    e4[kq] = 0;   // e, v, idx are filled in by the redo pass
-                    v4[kq] = 0;
-                    idx = 0;
-                } else {
-                    kernel9_exact(wbuf + n * 9, y, s2, cbuf + n * 9, e4[kq], v4[kq], idx);
-                }
+                if (pos < redo_cap) redo[pos] = static_cast<unsigned short>(n);
+                else overflow |= 1u << kq;
+                e4[kq] = 0;
+                v4[kq] = 0;
+                idx = 0;
             }
             hist_add(hist, v4[kq]);
             i4 |= static_cast<unsigned>(idx) << (8 * kq);
@@ -679,6 +762,21 @@ __device__ __forceinline__ void channel_body_k9_fast(const LayerDesc &L, int m, 
         reinterpret_cast<int4 *>(ev)[Q] = make_int4(e4[0], e4[1], e4[2], e4[3]);
         reinterpret_cast<int4 *>(vv)[Q] = make_int4(v4[0], v4[1], v4[2], v4[3]);
         reinterpret_cast<unsigned *>(vi)[Q] = i4;
+        if (overflow) {   // redo list full (tiny N or massive ties): do them here
+#pragma unroll 1
+            for (int kq = 0; kq < 4; ++kq) {
+                if (overflow & (1u << kq)) {
+                    const int n = 4 * Q + kq;
+                    int e1, v, idx;
+                    kernel9_exact(wbuf + n * 9, y, s2, cbuf + n * 9, e1, v, idx);
+                    ev[n] = e1;
+                    vv[n] = v;
+                    vi[n] = static_cast<unsigned char>(idx);
+                    hist_add(hist, v);
+                    esum += e1;
+                }
+            }
+        }
     }
     G.sync();
     {   // kernels handed back by the fast selection, redone exactly, densely over the group
@@ -834,20 +932,25 @@ __device__ __forceinline__ void channel_body_k9_fast(const LayerDesc &L, int m, 
         G.sync();
     }
 
-    // ---- codes (bias removed), scale, channel error
+    // ---- codes, scale, channel error
     int8_t *cg = L.codes + static_cast<size_t>(m) * NK;
+    if ((reinterpret_cast<uintptr_t>(cg) & 15) == 0 && (NK & 15) == 0) {
+        if (G.t == 0) {   // one bulk asynchronous copy of the staged codes
+            bulk_store(cg, cbuf, static_cast<unsigned>(NK));
+            L.scales[m] = s;
+            if (L.cerr) L.cerr[m] = __fmul_rn(__ll2float_rn(ec), 0x1p-30f);
+            bulk_store_wait();   // shared memory must stay intact until it has been read
+        }
+        return;
+    }
     if ((reinterpret_cast<uintptr_t>(cg) & 15) == 0) {
         const int nv = NK >> 4;
         const int4 *src = reinterpret_cast<const int4 *>(cbuf);
         int4 *dst = reinterpret_cast<int4 *>(cg);
-        for (int i = G.t; i < nv; i += G.g) {
-            int4 t = src[i];
-            t.x ^= 0x80808080; t.y ^= 0x80808080; t.z ^= 0x80808080; t.w ^= 0x80808080;
-            __stcs(dst + i, t);
-        }
-        for (int i = (nv << 4) + G.t; i < NK; i += G.g) cg[i] = static_cast<int8_t>(cbuf[i] ^ 0x80);
+        for (int i = G.t; i < nv; i += G.g) __stcs(dst + i, src[i]);
+        for (int i = (nv << 4) + G.t; i < NK; i += G.g) cg[i] = static_cast<int8_t>(cbuf[i]);
     } else {
-        for (int i = G.t; i < NK; i += G.g) cg[i] = static_cast<int8_t>(cbuf[i] ^ 0x80);
+        for (int i = G.t; i < NK; i += G.g) cg[i] = static_cast<int8_t>(cbuf[i]);
     }
     if (G.t == 0) {
         L.scales[m] = s;
@@ -875,6 +978,7 @@ squant_model_kernel(const LayerDesc *__restrict__ layers, const Item *__restrict
     if (m >= L.M) return;   // the whole group leaves together; it shares no barrier with others
     unsigned char *slice = smem + static_cast<size_t>(gi) * L.slice_bytes;
     const float s = stage_channel(L, m, G, slice, qmax);
+    if (s == 0.0f) return;   // staging wait ran out (status word set); nothing is written
     if (L.K == 1) {
         channel_body<1>(L, m, G, slice, s, mode);
     } else if (L.K == 9) {

@@ -24,8 +24,8 @@ def test_library_exports_every_declared_symbol():
 
 def test_strerror_covers_all_codes():
     lib = sq.load_library()
-    texts = {lib.squant_strerror(c).decode() for c in range(0, -10, -1)}
-    assert len(texts) == 10 and all(texts)
+    texts = {lib.squant_strerror(c).decode() for c in range(0, -11, -1)}
+    assert len(texts) == 11 and all(texts)
     assert "unknown" in lib.squant_strerror(-99).decode()
 
 

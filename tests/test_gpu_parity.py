@@ -20,7 +20,7 @@ def run_gpu(ws, bits, mode, flags=sq.FLAG_NARROW_RANGE):
     for b in bufs:   # poison the outputs so that an unwritten element cannot pass
         b.codes.fill_(-128); b.scales.fill_(float("nan")); b.kernel_err.fill_(float("nan")); b.channel_err.fill_(float("nan"))
     sq.squant_quantize_model(bufs, bits=bits, mode=mode, flags=flags)
-    torch.cuda.synchronize()
+    sq.squant_device_status()      # synchronises; raises if a kernel gave up a bounded wait
     return bufs
 
 
