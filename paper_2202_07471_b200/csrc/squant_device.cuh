@@ -391,9 +391,13 @@ __device__ __forceinline__ void squant_e_fast(float w, float y, float s2, unsign
 }
 
 // Exact SQuant-K + Algorithm 3 on one 3x3 kernel from its weights in shared memory; codes are
-// written as bytes.  Used for the few kernels the fast selection hands back.
-__device__ __forceinline__ void kernel9_exact(const float *wk, float y, float s2, unsigned char *cb,
-                                              int &e_out, int &v_out, int &idx_out)
+// written as bytes.  Used for the few kernels the fast selection hands back; kept out of line so
+// that the common path stays small.
+struct KernelOut {
+    int e, v, idx;
+};
+
+__device__ __noinline__ KernelOut kernel9_exact(const float *wk, float y, float s2, unsigned char *cb)
 {
     int P[9], q[9];
     long long e = 0;
@@ -439,14 +443,16 @@ __device__ __forceinline__ void kernel9_exact(const float *wk, float y, float s2
     }
 #pragma unroll
     for (int i = 0; i < 9; ++i) cb[i] = static_cast<unsigned char>(q[i]);
-    e_out = static_cast<int>(e);
-    v_out = v;
-    idx_out = idx;
+    KernelOut o;
+    o.e = static_cast<int>(e);
+    o.v = v;
+    o.idx = idx;
+    return o;
 }
 
 // Fast SQuant-K + Algorithm 3 on one 3x3 kernel whose exact perturbations Pf[0..8] (floats, in
-// 2^-30 units, before the conversion to integers) are in registers and whose code bytes
-// are already staged at cb.  Straight-line on purpose: every lane runs the same instructions and
+// 2^-30 units, before the conversion to integers) are in registers and whose code bytes are
+// already staged at cb.  Straight-line on purpose: every lane runs the same instructions and
 // the rare hand-back to kernel9_exact is a returned flag.
 //
 // Sign, flip count and Over/Under come from a float sum of the perturbations.  That sum is
@@ -458,10 +464,10 @@ __device__ __forceinline__ void kernel9_exact(const float *wk, float y, float s2
 // The exact |e| is still summed in integers (mod 2^32) for the error sum that is emitted.
 //
 // Selection: keys are the sign-normalised integer perturbations with the element index folded
-// into their low four bits, (P & ~15) | (15 - i), so the three largest can be tracked by value
+// into their low four bits, (P & ~15) | (15 - i), so the four largest can be tracked by value
 // alone and carry their positions.  This orders by (P >> 4, index); it equals Algorithm 2's
 // order (P, index) whenever the truncated values of neighbouring ranks differ, which is checked.
-// Handled: j = 0 (k = 0), j = 1 (k = 1, Over), j = 2 (k = 1, Under), j = 3 (k = 2, Over).
+// Handled: j = 0..5, i.e. k = 0, 1, 2 and k = 3 when it is Over SQuant.
 __device__ __forceinline__ bool kernel9_fast(const float (&Pf)[9], const float *wk, float y, float s2,
                                              unsigned char *cb, int &e_out, int &v_out, int &idx_out)
 {
@@ -473,7 +479,7 @@ __device__ __forceinline__ bool kernel9_fast(const float (&Pf)[9], const float *
     const float v = __fmul_rn(fabsf(ef), 0x1p-29f);
     const bool near = fabsf(__fsub_rn(v, rintf(v))) < 0x1p-17f;
     const int j = __float2int_rd(v);
-    int m1 = 0, m2 = 0, m3 = 0;
+    int m1 = 0, m2 = 0, m3 = 0, m4 = 0;
     unsigned eabs = 0;   // |e| mod 2^32
 #pragma unroll
     for (int i = 0; i < 9; ++i) {
@@ -484,23 +490,29 @@ __device__ __forceinline__ bool kernel9_fast(const float (&Pf)[9], const float *
         m1 = max(m1, key);
         const int u = min(m2, t);
         m2 = max(m2, t);
+        const int x = min(m3, u);
         m3 = max(m3, u);
+        m4 = max(m4, x);
     }
-    const bool d12 = (m1 >> 4) > (m2 >> 4), d23 = (m2 >> 4) > (m3 >> 4);
+    const bool d12 = (m1 >> 4) > (m2 >> 4), d23 = (m2 >> 4) > (m3 >> 4), d34 = (m3 >> 4) > (m4 >> 4);
     const bool zero = near & (j == 0) & (eabs == 0u);   // e == 0: no flips, no candidate
-    const bool ok = zero | (!near & d12 & ((j <= 1) | (d23 & (j <= 3))));
-    // ok with j >= 1 implies m1 >= 16, ok with j >= 2 implies m2 >= 16: the indices below are 0..8
+    const bool ok = zero | (!near & d12 & ((j <= 1) | (d23 & ((j <= 3) | (d34 & (j <= 5))))));
+    // ok with j >= 1 implies m1 >= 16, with j >= 2 m2 >= 16, with j >= 4 m3 >= 16: indices are 0..8
     if (ok & (j >= 1)) {
-        const int i1 = 15 - (m1 & 15);
+        const int i1 = ~m1 & 15;   // = 15 - (m1 & 15)
         cb[i1] = static_cast<unsigned char>(cb[i1] - sgn);
     }
-    if (ok & (j == 3)) {
-        const int i2 = 15 - (m2 & 15);
+    if (ok & (j >= 3)) {
+        const int i2 = ~m2 & 15;
         cb[i2] = static_cast<unsigned char>(cb[i2] - sgn);
     }
+    if (ok & (j == 5)) {
+        const int i3 = ~m3 & 15;
+        cb[i3] = static_cast<unsigned char>(cb[i3] - sgn);
+    }
     // candidate: Over (j odd) -> the k-th (last flipped), Under -> the (k+1)-th
-    const int mc = (j <= 1) ? m1 : m2;
-    const int idx = 15 - (mc & 15);   // at most 15: stays inside the staged channel
+    const int mc = (j <= 1) ? m1 : ((j <= 3) ? m2 : m3);
+    const int idx = ~mc & 15;   // at most 15: stays inside the staged channel
     unsigned tb;
     float Pcf;
     squant_e_fastf(wk[idx], y, s2, tb, Pcf);   // exact value of the candidate's perturbation
@@ -530,6 +542,14 @@ __device__ __forceinline__ float stage_channel(const LayerDesc &L, int m, const 
     int *flag = reinterpret_cast<int *>(red + 200);
     const float *wg = L.w + static_cast<size_t>(m) * NK;
     float amax = 0.0f;
+    {   // channel-step scratch starts at zero; the barriers below publish it
+        int *hist = reinterpret_cast<int *>(slice + L.off_hist);
+        for (int i = G.t; i < kHistBins; i += G.g) hist[i] = 0;
+        if (G.t == 0) {
+            reinterpret_cast<int *>(red + 128)[5] = 0;                    // boundary-list count
+            *reinterpret_cast<unsigned long long *>(red + 208) = 0ull;   // channel-sum accumulator
+        }
+    }
     if ((reinterpret_cast<uintptr_t>(wg) & 15) == 0 && (NK & 3) == 0) {
         if (G.t == 0) {
             *flag = 0;
@@ -676,22 +696,22 @@ __device__ __forceinline__ void channel_body(const LayerDesc &L, int m, const Gr
 // Needs K = 9, N a multiple of 4, SQuant-K in the mode mask and 2^-60 <= s <= 2^60.
 // A thread owns four consecutive kernels = 36 consecutive weights: nine conflict-free 128-bit
 // shared loads in, nine conflict-free 32-bit stores of packed code bytes out; flips are byte
-// read-modify-writes on the staged codes.
+// read-modify-writes on the staged codes.  Kernel error sums are written as soon as SQuant-K is
+// done; SQuant-C later patches the few kernels it flips.
 //
-// SQuant-C here needs ONE histogram, filled while the kernels are processed: bin = |v| >> 22 of
-// each kernel's candidate, positive and negative candidates counted in the two halves of one
-// 32-bit word.  Once the channel sum (hence the sign and k_c) is known, a warp scans the
-// histogram of that sign for the boundary bin; kernels above it are flipped, the few inside it
-// are collected in a list and ranked exactly (|v| descending, kernel index ascending).  A boundary
-// bin too crowded for the list (massive ties) falls back to the general radix select.
+// SQuant-C needs ONE histogram, filled while the kernels are processed: bin = |v| >> 22 of each
+// kernel's candidate, positive and negative candidates counted in the two halves of one 32-bit
+// word.  Once the channel sum (hence the sign and k_c) is known, one warp scans the histogram
+// of that sign for the boundary bin;
+// kernels above it are flipped, the few inside it are collected in a list and ranked exactly
+// (|v| descending, kernel index ascending).  A boundary bin too crowded for the list (massive
+// ties) falls back to the general radix select.
 constexpr int kListCap = 256;
 
 __device__ __forceinline__ void hist_add(int *hist, int v)
 {
-    if (v != 0) {
-        const int a = v > 0 ? v : -v;
-        atomicAdd(&hist[hist_slot(a >> 22)], v > 0 ? 1 : 0x10000);
-    }
+    const int a = v < 0 ? -v : v;                           // < 2^30: bin < 256
+    atomicAdd(&hist[a >> 22], (v > 0 ? 1 : 0) | (v < 0 ? 0x10000 : 0));
 }
 
 __device__ __forceinline__ void channel_body_k9_fast(const LayerDesc &L, int m, const Group &G,
@@ -702,17 +722,14 @@ __device__ __forceinline__ void channel_body_k9_fast(const LayerDesc &L, int m, 
     unsigned char *cbuf = slice + L.off_codes;
     int *ev = reinterpret_cast<int *>(slice + L.off_ev);
     int *vv = reinterpret_cast<int *>(slice + L.off_vv);
-    unsigned char *vi = slice + L.off_vi;                       // N index bytes, then the redo list
-    unsigned short *redo = reinterpret_cast<unsigned short *>(vi + N);
-    const int redo_cap = N >> 1;
+    unsigned char *vi = slice + L.off_vi;
     int *hist = reinterpret_cast<int *>(slice + L.off_hist);
     unsigned char *red = slice + L.off_red;
-    int *bc = reinterpret_cast<int *>(red + 128);               // [0..3] scan result, [4] redo count, [5] list count
+    int *bc = reinterpret_cast<int *>(red + 128);               // [0..3] radix-select scratch, [5] list count
+    unsigned long long *acc = reinterpret_cast<unsigned long long *>(red + 208);
     int2 *blist = reinterpret_cast<int2 *>(slice);              // boundary list: reuses the weights' space
-
-    for (int i = G.t; i < kHistBins; i += G.g) hist[i] = 0;
-    if (G.t == 0) { bc[4] = 0; bc[5] = 0; }
-    G.sync();
+    float *kerr = L.kerr ? L.kerr + static_cast<size_t>(m) * N : nullptr;
+    const bool kvec = (reinterpret_cast<uintptr_t>(kerr) & 15) == 0;
 
     const float s2 = __fmul_rn(s, 0x1p-30f);
     const float y = __frcp_rn(s2);
@@ -721,82 +738,73 @@ __device__ __forceinline__ void channel_body_k9_fast(const LayerDesc &L, int m, 
     for (int Q = G.t; Q < quads; Q += G.g) {
         const float4 *src = reinterpret_cast<const float4 *>(wbuf) + Q * 9;
         unsigned *dst = reinterpret_cast<unsigned *>(cbuf) + Q * 9;
-        float w[36];
-#pragma unroll
-        for (int j = 0; j < 9; ++j) {
-            const float4 t = src[j];
-            w[4 * j] = t.x; w[4 * j + 1] = t.y; w[4 * j + 2] = t.z; w[4 * j + 3] = t.w;
-        }
         float P[36];
 #pragma unroll
         for (int j = 0; j < 9; ++j) {
+            const float4 w = src[j];
             unsigned t0, t1, t2, t3;
-            squant_e_fastf(w[4 * j], y, s2, t0, P[4 * j]);
-            squant_e_fastf(w[4 * j + 1], y, s2, t1, P[4 * j + 1]);
-            squant_e_fastf(w[4 * j + 2], y, s2, t2, P[4 * j + 2]);
-            squant_e_fastf(w[4 * j + 3], y, s2, t3, P[4 * j + 3]);
+            squant_e_fastf(w.x, y, s2, t0, P[4 * j]);
+            squant_e_fastf(w.y, y, s2, t1, P[4 * j + 1]);
+            squant_e_fastf(w.z, y, s2, t2, P[4 * j + 2]);
+            squant_e_fastf(w.w, y, s2, t3, P[4 * j + 3]);
             dst[j] = __byte_perm(__byte_perm(t0, t1, 0x0040), __byte_perm(t2, t3, 0x0040), 0x5410);
         }
         int e4[4], v4[4];
-        unsigned i4 = 0, overflow = 0;
+        unsigned i4 = 0, again = 0;
+        const float *wq = wbuf + Q * 36;
+        unsigned char *cq = cbuf + Q * 36;
 #pragma unroll
         for (int kq = 0; kq < 4; ++kq) {
             float Pk[9];
 #pragma unroll
             for (int i = 0; i < 9; ++i) Pk[i] = P[9 * kq + i];
-            const int n = 4 * Q + kq;
             int idx;
-            const bool again = kernel9_fast(Pk, wbuf + n * 9, y, s2, cbuf + n * 9, e4[kq], v4[kq], idx);
-            if (again) {   // e, v, idx are filled in by the redo pass
-                const int pos = atomicAdd(&bc[4], 1);
-                if (pos < redo_cap) redo[pos] = static_cast<unsigned short>(n);
-                else overflow |= 1u << kq;
+            if (kernel9_fast(Pk, wq + 9 * kq, y, s2, cq + 9 * kq, e4[kq], v4[kq], idx)) {
+                again |= 1u << kq;   // redone exactly below
                 e4[kq] = 0;
                 v4[kq] = 0;
                 idx = 0;
             }
             hist_add(hist, v4[kq]);
             i4 |= static_cast<unsigned>(idx) << (8 * kq);
-            esum += e4[kq];
         }
+        esum += static_cast<long long>(e4[0] + e4[1]) + (e4[2] + e4[3]);   // pairs fit 32 bits
         reinterpret_cast<int4 *>(ev)[Q] = make_int4(e4[0], e4[1], e4[2], e4[3]);
         reinterpret_cast<int4 *>(vv)[Q] = make_int4(v4[0], v4[1], v4[2], v4[3]);
         reinterpret_cast<unsigned *>(vi)[Q] = i4;
-        if (overflow) {   // redo list full (tiny N or massive ties): do them here
+        if (kerr) {
+            float4 f;
+            f.x = __fmul_rn(__int2float_rn(e4[0]), 0x1p-30f);
+            f.y = __fmul_rn(__int2float_rn(e4[1]), 0x1p-30f);
+            f.z = __fmul_rn(__int2float_rn(e4[2]), 0x1p-30f);
+            f.w = __fmul_rn(__int2float_rn(e4[3]), 0x1p-30f);
+            if (kvec) __stcs(reinterpret_cast<float4 *>(kerr) + Q, f);
+            else { kerr[4 * Q] = f.x; kerr[4 * Q + 1] = f.y; kerr[4 * Q + 2] = f.z; kerr[4 * Q + 3] = f.w; }
+        }
+        if (again) {   // rare: kernels the fast selection handed back
 #pragma unroll 1
             for (int kq = 0; kq < 4; ++kq) {
-                if (overflow & (1u << kq)) {
+                if (again & (1u << kq)) {
                     const int n = 4 * Q + kq;
-                    int e1, v, idx;
-                    kernel9_exact(wbuf + n * 9, y, s2, cbuf + n * 9, e1, v, idx);
-                    ev[n] = e1;
-                    vv[n] = v;
-                    vi[n] = static_cast<unsigned char>(idx);
-                    hist_add(hist, v);
-                    esum += e1;
+                    const KernelOut o = kernel9_exact(wbuf + n * 9, y, s2, cbuf + n * 9);
+                    ev[n] = o.e;
+                    vv[n] = o.v;
+                    vi[n] = static_cast<unsigned char>(o.idx);
+                    if (kerr) kerr[n] = __fmul_rn(__int2float_rn(o.e), 0x1p-30f);
+                    hist_add(hist, o.v);
+                    esum += o.e;
                 }
             }
         }
     }
-    G.sync();
-    {   // kernels handed back by the fast selection, redone exactly, densely over the group
-        const int nredo = min(bc[4], redo_cap);
-        for (int i = G.t; i < nredo; i += G.g) {
-            const int n = redo[i];
-            int e1, v, idx;
-            kernel9_exact(wbuf + n * 9, y, s2, cbuf + n * 9, e1, v, idx);
-            ev[n] = e1;
-            vv[n] = v;
-            vi[n] = static_cast<unsigned char>(idx);
-            hist_add(hist, v);
-            esum += e1;
-        }
-    }
+    // channel sum: warp shuffle, then one shared atomic per warp
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) esum += __shfl_xor_sync(kFull, esum, o);
+    if ((G.t & 31) == 0) atomicAdd(acc, static_cast<unsigned long long>(esum));
+    G.sync();   // per-kernel data, histogram and channel sum visible
+    long long ec = static_cast<long long>(*acc);
 
-    // ---- SQuant-C: channel sum, boundary bin
-    long long ec = 0;
-    if ((mode & 4u) || L.cerr) ec = group_sum(G, esum, red);   // barrier: per-kernel data, histogram visible
-    else G.sync();
+    // ---- SQuant-C: boundary bin of the candidate histogram
     int sgn_c = 0, k_eff = 0;
     int t_all = 0x7fffffff;     // candidates with v * sgn_c >= t_all are flipped outright
     int t_list = 0x7fffffff;    // those in [t_list, t_all) go to the boundary list
@@ -808,11 +816,13 @@ __device__ __forceinline__ void channel_body_k9_fast(const LayerDesc &L, int m, 
         const long long abs_e = ec > 0 ? ec : -ec;
         const int kc = flip_count(abs_e);
         if (kc > 0) {
-            if (G.t < 32) {
+            if (G.t < 32) {   // the group's first warp scans, highest bins first
                 const int lane = G.t, grp = 31 - lane, sh = sgn_c > 0 ? 0 : 16;
-                int c[8], s8 = 0;
-#pragma unroll
-                for (int j = 0; j < 8; ++j) { c[j] = (hist[(j << 5) | grp] >> sh) & 0xffff; s8 += c[j]; }
+                const int4 h0 = reinterpret_cast<const int4 *>(hist)[2 * grp];
+                const int4 h1 = reinterpret_cast<const int4 *>(hist)[2 * grp + 1];
+                const int c[8] = {(h0.x >> sh) & 0xffff, (h0.y >> sh) & 0xffff, (h0.z >> sh) & 0xffff, (h0.w >> sh) & 0xffff,
+                                  (h1.x >> sh) & 0xffff, (h1.y >> sh) & 0xffff, (h1.z >> sh) & 0xffff, (h1.w >> sh) & 0xffff};
+                const int s8 = ((c[0] + c[1]) + (c[2] + c[3])) + ((c[4] + c[5]) + (c[6] + c[7]));
                 int incl = s8;
 #pragma unroll
                 for (int o = 1; o < 32; o <<= 1) {
@@ -820,94 +830,70 @@ __device__ __forceinline__ void channel_body_k9_fast(const LayerDesc &L, int m, 
                     if (lane >= o) incl += t;
                 }
                 const int total = __shfl_sync(kFull, incl, 31);
-                const int want = min(kc, total);
-                const unsigned bal = __ballot_sync(kFull, incl >= want);
-                if (want <= 0) {
+                const int wnt = min(kc, total);
+                const unsigned bal = __ballot_sync(kFull, incl >= wnt);
+                if (wnt <= 0) {
                     if (lane == 0) { bc[0] = -1; bc[1] = 0; bc[2] = 0; bc[3] = 0; }
                 } else if (lane == __ffs(bal) - 1) {
-                    int cum = incl - s8, b = -1, cnt = 0;
+                    int bb = -1, cnt = 0, cum = incl - s8;
 #pragma unroll
                     for (int j = 7; j >= 0; --j) {
-                        if (b < 0) {
-                            if (cum + c[j] >= want) { b = grp * 8 + j; cnt = c[j]; }
+                        if (bb < 0) {
+                            if (cum + c[j] >= wnt) { bb = grp * 8 + j; cnt = c[j]; }
                             else cum += c[j];
                         }
                     }
-                    bc[0] = b; bc[1] = want - cum; bc[2] = cnt; bc[3] = want;
+                    bc[0] = bb; bc[1] = wnt - cum; bc[2] = cnt; bc[3] = wnt;
                 }
             }
             G.sync();
-            const int b = bc[0];
+            const int b = bc[0], want = bc[3];
             rem = bc[1];
             cb = bc[2];
-            k_eff = bc[3];
-            if (b >= 0) {
+            k_eff = want;
+            if (want > 0) {
                 if (cb == rem) {                 // whole boundary bin flipped
-                    t_all = max(b << 22, 1);   // 0 is "no candidate"
+                    t_all = max(b << 22, 1);     // 0 is "no candidate"
                 } else if (cb <= kListCap) {     // rank the boundary bin exactly
                     t_all = (b + 1) << 22;       // b + 1 = 256 gives 2^30, above every |v|
                     t_list = max(b << 22, 1);
                 } else {                         // crowded bin: general radix select on 48-bit keys
                     wide = true;
-                    G.sync();                    // everyone has read bc before the select reuses it
+                    G.sync();                    // everyone has read the scan result
                     k_eff = select_threshold(G, vv, N, sgn_c, kc, hist, bc, T64);
                 }
-            } else {
-                k_eff = 0;
             }
             ec -= static_cast<long long>(sgn_c) * k_eff * kOne;
         }
     }
 
-    // ---- apply the channel flips, emit the kernels' error sums (four kernels per thread)
-    float *kerr = L.kerr ? L.kerr + static_cast<size_t>(m) * N : nullptr;
+    // ---- flip the selected kernels' candidates and patch their error sums (rare per kernel)
     const bool listing = t_list != 0x7fffffff;
-    if (k_eff > 0 || kerr) {
-        const bool vec = kerr && !listing && (reinterpret_cast<uintptr_t>(kerr) & 15) == 0;
+    if (k_eff > 0) {
+        const int t_min = wide ? 1 : min(t_all, t_list);
         for (int Q = G.t; Q < quads; Q += G.g) {
-            const int4 e4 = reinterpret_cast<const int4 *>(ev)[Q];
-            int e[4] = {e4.x, e4.y, e4.z, e4.w};
-            bool listed[4] = {false, false, false, false};
-            if (k_eff > 0) {
-                const int4 v4 = reinterpret_cast<const int4 *>(vv)[Q];
-                const int v[4] = {v4.x, v4.y, v4.z, v4.w};
-                const unsigned i4 = reinterpret_cast<const unsigned *>(vi)[Q];
+            const int4 v4 = reinterpret_cast<const int4 *>(vv)[Q];
+            const int v[4] = {v4.x, v4.y, v4.z, v4.w};
 #pragma unroll
-                for (int kq = 0; kq < 4; ++kq) {
+            for (int kq = 0; kq < 4; ++kq) {
+                const int a = v[kq] * sgn_c;
+                if (a >= t_min) {
                     const int n = 4 * Q + kq;
-                    const int a = v[kq] * sgn_c;
                     bool take;
                     if (wide) {
-                        const unsigned long long ck = cand_key(v[kq], sgn_c, n);
-                        take = ck != 0 && ck >= T64;
+                        take = cand_key(v[kq], sgn_c, n) >= T64;
                     } else {
                         take = a >= t_all;
-                        if (!take && a >= t_list) {
-                            listed[kq] = true;
+                        if (!take) {
                             const int pos = atomicAdd(&bc[5], 1);
                             if (pos < kListCap) blist[pos] = make_int2(a, n);
                         }
                     }
                     if (take) {
-                        e[kq] -= sgn_c * kOne;
-                        unsigned char *bp = cbuf + n * 9 + ((i4 >> (8 * kq)) & 255u);
+                        unsigned char *bp = cbuf + n * 9 + vi[n];
                         *bp = static_cast<unsigned char>(*bp - sgn_c);
+                        if (kerr) kerr[n] = __fmul_rn(__int2float_rn(ev[n] - sgn_c * kOne), 0x1p-30f);
                     }
-                }
-            }
-            if (kerr) {
-                float4 f;
-                f.x = __fmul_rn(__int2float_rn(e[0]), 0x1p-30f);
-                f.y = __fmul_rn(__int2float_rn(e[1]), 0x1p-30f);
-                f.z = __fmul_rn(__int2float_rn(e[2]), 0x1p-30f);
-                f.w = __fmul_rn(__int2float_rn(e[3]), 0x1p-30f);
-                if (vec) {
-                    __stcs(reinterpret_cast<float4 *>(kerr) + Q, f);
-                } else {   // listed kernels are written by the ranking step below
-                    if (!listed[0]) kerr[4 * Q] = f.x;
-                    if (!listed[1]) kerr[4 * Q + 1] = f.y;
-                    if (!listed[2]) kerr[4 * Q + 2] = f.z;
-                    if (!listed[3]) kerr[4 * Q + 3] = f.w;
                 }
             }
         }
@@ -921,13 +907,11 @@ __device__ __forceinline__ void channel_body_k9_fast(const LayerDesc &L, int m, 
                 const int2 o = blist[j];
                 rank += (o.x > me.x || (o.x == me.x && o.y < me.y)) ? 1 : 0;
             }
-            int e1 = ev[me.y];
             if (rank < rem) {
-                e1 -= sgn_c * kOne;
                 unsigned char *bp = cbuf + me.y * 9 + vi[me.y];
                 *bp = static_cast<unsigned char>(*bp - sgn_c);
+                if (kerr) kerr[me.y] = __fmul_rn(__int2float_rn(ev[me.y] - sgn_c * kOne), 0x1p-30f);
             }
-            if (kerr) kerr[me.y] = __fmul_rn(__int2float_rn(e1), 0x1p-30f);
         }
         G.sync();
     }
