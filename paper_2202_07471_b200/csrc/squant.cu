@@ -97,7 +97,31 @@ int validate(const squant_layer *layers, int32_t n_layers, const squant_options 
     return SQUANT_OK;
 }
 
-// Shared-memory slice of one channel group and the grouped work list.
+// Device-side descriptor of one layer: group size and the layout of a group's shared-memory
+// slice.  Returns the dynamic shared memory one CTA needs for this layer.
+int64_t layout_layer(const squant_layer &l, LayerDesc &d)
+{
+    d.w = l.w; d.codes = l.codes; d.scales = l.scales; d.kerr = l.kernel_err; d.cerr = l.channel_err;
+    d.M = l.cout; d.N = l.cin; d.K = l.kh * l.kw; d.NK = d.N * d.K;
+    d.g = group_size(d.NK);
+    d.g_shift = 0;
+    while ((1 << d.g_shift) < d.g) ++d.g_shift;
+    int off = align16(4 * d.NK);              // staged weights
+    d.off_codes = off; off += align16(d.NK);  // staged codes
+    if (d.K == 1) {                           // 1x1: perturbations overwrite the weights
+        d.off_ev = 0; d.off_vv = 0; d.off_vi = 0;
+    } else {
+        d.off_ev = off; off += align16(4 * d.N);
+        d.off_vv = off; off += align16(4 * d.N);
+        d.off_vi = off; off += align16(2 * d.N);
+    }
+    d.off_hist = off; off += 4 * sq::kHistBins;
+    d.off_red = off; off += 256;
+    d.slice_bytes = off;
+    return static_cast<int64_t>(sq::kCtaThreads / d.g) * off;
+}
+
+// Work list in a table (global-memory variant): CTA-sized items, heaviest first.
 int build_plan(const squant_layer *layers, int32_t n_layers, const squant_options &o, int max_smem,
                HostPlan &p)
 {
@@ -108,27 +132,9 @@ int build_plan(const squant_layer *layers, int32_t n_layers, const squant_option
     struct Batch { int64_t work; int layer; int ch0; };
     std::vector<Batch> batches;
     for (int i = 0; i < n_layers; ++i) {
-        const squant_layer &l = layers[i];
         LayerDesc &d = p.layers[i];
-        d.w = l.w; d.codes = l.codes; d.scales = l.scales; d.kerr = l.kernel_err; d.cerr = l.channel_err;
-        d.M = l.cout; d.N = l.cin; d.K = l.kh * l.kw; d.NK = d.N * d.K;
-        d.g = group_size(d.NK);
-        d.g_shift = 0;
-        while ((1 << d.g_shift) < d.g) ++d.g_shift;
-        int off = align16(4 * d.NK);              // staged weights
-        d.off_codes = off; off += align16(d.NK);  // staged codes
-        if (d.K == 1) {                           // 1x1: perturbations overwrite the weights
-            d.off_ev = 0; d.off_vv = 0; d.off_vi = 0;
-        } else {
-            d.off_ev = off; off += align16(4 * d.N);
-            d.off_vv = off; off += align16(4 * d.N);
-            d.off_vi = off; off += align16(2 * d.N);
-        }
-        d.off_hist = off; off += 4 * sq::kHistBins;
-        d.off_red = off; off += 256;
-        d.slice_bytes = off;
+        const int64_t cta_smem = layout_layer(layers[i], d);
         const int groups = sq::kCtaThreads / d.g;
-        const int64_t cta_smem = static_cast<int64_t>(groups) * off;
         if (cta_smem > max_smem) return SQUANT_ERR_TOO_WIDE;
         if (cta_smem > p.smem_bytes) p.smem_bytes = static_cast<int>(cta_smem);
         for (int c = 0; c < d.M; c += groups) {
@@ -144,17 +150,66 @@ int build_plan(const squant_layer *layers, int32_t n_layers, const squant_option
     return SQUANT_OK;
 }
 
-// A plan resident on one device, keyed by the exact descriptors and options.
-struct DevicePlan {
-    int device = -1;
-    std::string key;
-    void *table = nullptr;   // LayerDesc[n_layers] followed by Item[n_items]
-    int n_layers = 0, n_items = 0, smem_bytes = 0, qmax = 0;
+// Launch tables for the parameter-space variant: layers ordered by the work of one of their
+// CTAs (heaviest first, so the tail of the launch is made of light CTAs), at most
+// kMaxParamLayers per launch.
+struct ParamPlan {
+    std::vector<sq::LaunchTable> tables;
+    std::vector<int> grids;
+    int smem_bytes = 0, qmax = 0;
     unsigned mode = 0;
 };
 
-std::list<DevicePlan> g_plans;              // most recently used first
-std::vector<int> g_smem_limit_by_device;   // opt-in limit set on the kernel, per device
+int build_param_plan(const squant_layer *layers, int32_t n_layers, const squant_options &o,
+                     int max_smem, ParamPlan &p)
+{
+    p.qmax = (1 << (o.bits - 1)) - 1;
+    p.mode = o.mode;
+    p.smem_bytes = 0;
+    std::vector<LayerDesc> descs(n_layers);
+    std::vector<int> order(n_layers);
+    for (int i = 0; i < n_layers; ++i) {
+        const int64_t cta_smem = layout_layer(layers[i], descs[i]);
+        if (cta_smem > max_smem) return SQUANT_ERR_TOO_WIDE;
+        if (cta_smem > p.smem_bytes) p.smem_bytes = static_cast<int>(cta_smem);
+        order[i] = i;
+    }
+    auto cta_work = [&](int i) {
+        const LayerDesc &d = descs[i];
+        const int64_t groups = sq::kCtaThreads / d.g;
+        return (groups < d.M ? groups : d.M) * static_cast<int64_t>(d.NK);
+    };
+    std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return cta_work(a) > cta_work(b); });
+    for (int base = 0; base < n_layers; base += sq::kMaxParamLayers) {
+        const int n = (n_layers - base < sq::kMaxParamLayers) ? n_layers - base : sq::kMaxParamLayers;
+        p.tables.emplace_back();
+        sq::LaunchTable &t = p.tables.back();
+        std::memset(&t, 0, sizeof(t));
+        t.n_layers = n;
+        int items = 0;
+        for (int j = 0; j < n; ++j) {
+            const LayerDesc &d = descs[order[base + j]];
+            const int groups = sq::kCtaThreads / d.g;
+            t.layers[j] = d;
+            t.first_item[j] = items;
+            items += (d.M + groups - 1) / groups;
+        }
+        for (int j = n; j <= sq::kMaxParamLayers; ++j) t.first_item[j] = items;
+        p.grids.push_back(items);
+    }
+    return SQUANT_OK;
+}
+
+// Launch tables are plain host data; the most recent ones are kept, keyed by the exact
+// descriptors and options, so that a repeated call only enqueues its kernel(s).
+struct CachedPlan {
+    int device = -1;
+    std::string key;
+    ParamPlan plan;
+};
+
+std::list<CachedPlan> g_plans;              // most recently used first
+std::vector<int> g_smem_limit_by_device;   // opt-in limit set on the kernels, per device
 
 std::string plan_key(const squant_layer *layers, int32_t n_layers, const squant_options &o)
 {
@@ -172,14 +227,15 @@ int device_smem_limit(int device, int &limit)
         SQ_CUDA(cudaDeviceGetAttribute(&v, cudaDevAttrMaxSharedMemoryPerBlockOptin, device));
         SQ_CUDA(cudaFuncSetAttribute(sq::squant_model_kernel,
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, v));
+        SQ_CUDA(cudaFuncSetAttribute(sq::squant_table_kernel,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, v));
         g_smem_limit_by_device[device] = v;
     }
     limit = g_smem_limit_by_device[device];
     return SQUANT_OK;
 }
 
-int get_plan(const squant_layer *layers, int32_t n_layers, const squant_options &o,
-             cudaStream_t stream, DevicePlan *&out)
+int get_plan(const squant_layer *layers, int32_t n_layers, const squant_options &o, const ParamPlan *&out)
 {
     int device = 0;
     SQ_CUDA(cudaGetDevice(&device));
@@ -187,59 +243,32 @@ int get_plan(const squant_layer *layers, int32_t n_layers, const squant_options 
     for (auto it = g_plans.begin(); it != g_plans.end(); ++it) {
         if (it->device == device && it->key == key) {
             g_plans.splice(g_plans.begin(), g_plans, it);
-            out = &g_plans.front();
+            out = &g_plans.front().plan;
             return SQUANT_OK;
         }
     }
     int limit = 0;
     int rc = device_smem_limit(device, limit);
     if (rc) return rc;
-    HostPlan hp;
-    rc = build_plan(layers, n_layers, o, limit, hp);
+    CachedPlan cp;
+    cp.device = device;
+    cp.key = std::move(key);
+    rc = build_param_plan(layers, n_layers, o, limit, cp.plan);
     if (rc) return rc;
-    DevicePlan dp;
-    dp.device = device;
-    dp.key = std::move(key);
-    dp.n_layers = n_layers;
-    dp.n_items = static_cast<int>(hp.items.size());
-    dp.smem_bytes = hp.smem_bytes;
-    dp.qmax = hp.qmax;
-    dp.mode = hp.mode;
-    const size_t lbytes = sizeof(LayerDesc) * hp.layers.size();
-    const size_t ibytes = sizeof(Item) * hp.items.size();
-    if (lbytes + ibytes > 0) {
-        std::vector<unsigned char> host(lbytes + ibytes);
-        std::memcpy(host.data(), hp.layers.data(), lbytes);
-        std::memcpy(host.data() + lbytes, hp.items.data(), ibytes);
-        cudaError_t e = cudaMalloc(&dp.table, lbytes + ibytes);
-        if (e != cudaSuccess) return e == cudaErrorMemoryAllocation ? SQUANT_ERR_NOMEM : cuda_fail(e, "cudaMalloc");
-        e = cudaMemcpyAsync(dp.table, host.data(), lbytes + ibytes, cudaMemcpyHostToDevice, stream);
-        if (e == cudaSuccess) e = cudaStreamSynchronize(stream);   // host vector dies here
-        if (e != cudaSuccess) { cudaFree(dp.table); return cuda_fail(e, "plan upload"); }
-    }
-    if (g_plans.size() >= kMaxPlans) {
-        // The evicted table may still be read by an earlier launch: wait for the device first.
-        int cur = device;
-        cudaSetDevice(g_plans.back().device);
-        cudaDeviceSynchronize();
-        cudaFree(g_plans.back().table);
-        cudaSetDevice(cur);
-        g_plans.pop_back();
-    }
-    g_plans.push_front(std::move(dp));
-    out = &g_plans.front();
+    if (g_plans.size() >= kMaxPlans) g_plans.pop_back();
+    g_plans.push_front(std::move(cp));
+    out = &g_plans.front().plan;
     return SQUANT_OK;
 }
 
-int launch_plan(const DevicePlan &dp, cudaStream_t stream)
+int launch_plan(const ParamPlan &p, cudaStream_t stream)
 {
-    if (dp.n_items == 0) return SQUANT_OK;
-    const LayerDesc *dl = static_cast<const LayerDesc *>(dp.table);
-    const Item *di = reinterpret_cast<const Item *>(static_cast<const unsigned char *>(dp.table) +
-                                                    sizeof(LayerDesc) * dp.n_layers);
-    sq::squant_model_kernel<<<dp.n_items, sq::kCtaThreads, dp.smem_bytes, stream>>>(dl, di, dp.qmax, dp.mode);
-    SQ_CUDA(cudaGetLastError());
-    g_launches.fetch_add(1, std::memory_order_relaxed);
+    for (size_t c = 0; c < p.tables.size(); ++c) {
+        if (p.grids[c] == 0) continue;
+        sq::squant_model_kernel<<<p.grids[c], sq::kCtaThreads, p.smem_bytes, stream>>>(p.tables[c], p.qmax, p.mode);
+        SQ_CUDA(cudaGetLastError());
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+    }
     return SQUANT_OK;
 }
 
@@ -283,10 +312,10 @@ int squant_quantize_model(const squant_layer *layers, int32_t n_layers, const sq
     if (rc) return rc;
     if (n_layers == 0) return SQUANT_OK;
     std::lock_guard<std::mutex> lock(g_mutex);
-    DevicePlan *dp = nullptr;
-    rc = get_plan(layers, n_layers, o, static_cast<cudaStream_t>(cuda_stream), dp);
+    const ParamPlan *pp = nullptr;
+    rc = get_plan(layers, n_layers, o, pp);
     if (rc) return rc;
-    return launch_plan(*dp, static_cast<cudaStream_t>(cuda_stream));
+    return launch_plan(*pp, static_cast<cudaStream_t>(cuda_stream));
 }
 
 int squant_quantize_layer(const squant_layer *layer, const squant_options *opt, void *cuda_stream)
@@ -338,10 +367,10 @@ int squant_quantize_model_host(const squant_layer *layers, int32_t n_layers,
         dev[i].channel_err = l.channel_err ? reinterpret_cast<float *>(base + off[5 * i + 4]) : nullptr;
         SQ_CUDA(cudaMemcpyAsync(base + off[5 * i + 0], l.w, n * 4, cudaMemcpyHostToDevice, stream));
     }
-    DevicePlan *dp = nullptr;
-    rc = get_plan(dev.data(), n_layers, o, stream, dp);
+    const ParamPlan *pp = nullptr;
+    rc = get_plan(dev.data(), n_layers, o, pp);
     if (rc) return rc;
-    rc = launch_plan(*dp, stream);
+    rc = launch_plan(*pp, stream);
     if (rc) return rc;
     for (int i = 0; i < n_layers; ++i) {
         const squant_layer &l = layers[i];
@@ -387,7 +416,7 @@ int squant_quantize_layer_noalloc(const squant_layer *layer, const squant_option
     SQ_CUDA(cudaMemcpyAsync(table, g_noalloc_host, 256 + ibytes, cudaMemcpyHostToDevice, stream));
     const LayerDesc *dl = static_cast<const LayerDesc *>(table);
     const Item *di = reinterpret_cast<const Item *>(static_cast<const unsigned char *>(table) + 256);
-    sq::squant_model_kernel<<<static_cast<unsigned>(hp.items.size()), sq::kCtaThreads, hp.smem_bytes, stream>>>(
+    sq::squant_table_kernel<<<static_cast<unsigned>(hp.items.size()), sq::kCtaThreads, hp.smem_bytes, stream>>>(
         dl, di, hp.qmax, hp.mode);
     SQ_CUDA(cudaGetLastError());
     g_launches.fetch_add(1, std::memory_order_relaxed);
@@ -448,9 +477,6 @@ int squant_shutdown(void)
     std::lock_guard<std::mutex> lock(g_mutex);
     int cur = 0;
     const bool have = cudaGetDevice(&cur) == cudaSuccess;
-    for (auto &p : g_plans) {
-        if (p.table) { cudaSetDevice(p.device); cudaDeviceSynchronize(); cudaFree(p.table); }
-    }
     g_plans.clear();
     for (size_t d = 0; d < g_arenas.size(); ++d) {
         if (g_arenas[d].ptr) { cudaSetDevice(static_cast<int>(d)); cudaDeviceSynchronize(); cudaFree(g_arenas[d].ptr); }

@@ -42,6 +42,18 @@ struct Item {
     int32_t ch0;
 };
 
+// Everything a grouped launch needs, passed BY VALUE as a kernel parameter: the descriptors sit
+// in the constant bank, so a CTA finds its work without a single global load (and nothing has
+// to be allocated or uploaded).  Work items of layer l are the CTAs first_item[l] ..
+// first_item[l+1]-1; item i of a layer handles channels i * (512 / g) ... of it.
+constexpr int kMaxParamLayers = 96;
+struct LaunchTable {
+    int n_layers;
+    int pad;
+    int first_item[kMaxParamLayers + 1];
+    LayerDesc layers[kMaxParamLayers];
+};
+
 struct Group {
     int g;    // threads in the group
     int t;    // this thread's index inside the group
@@ -943,22 +955,20 @@ __device__ __forceinline__ void channel_body_k9_fast(const LayerDesc &L, int m, 
 }
 
 // ---------------------------------------------------------------- grouped launch
+// One CTA per work item.  The descriptor of the CTA's layer comes either from the launch table
+// in the kernel's parameter space (kParams) or from a table in global memory.
 #ifndef SQ_MIN_CTAS
 #define SQ_MIN_CTAS 2
 #endif
-__global__ void __launch_bounds__(kCtaThreads, SQ_MIN_CTAS)
-squant_model_kernel(const LayerDesc *__restrict__ layers, const Item *__restrict__ items, int qmax,
-                    unsigned mode)
+__device__ __forceinline__ void run_item(const LayerDesc &L, int ch0, unsigned char *smem, int qmax,
+                                         unsigned mode)
 {
-    extern __shared__ __align__(16) unsigned char smem[];
-    const Item it = items[blockIdx.x];
-    const LayerDesc L = layers[it.layer];
     Group G;
     G.g = L.g;
     G.t = threadIdx.x & (L.g - 1);
     const int gi = threadIdx.x >> L.g_shift;
     G.bar = 1 + gi;
-    const int m = it.ch0 + gi;
+    const int m = ch0 + gi;
     if (m >= L.M) return;   // the whole group leaves together; it shares no barrier with others
     unsigned char *slice = smem + static_cast<size_t>(gi) * L.slice_bytes;
     const float s = stage_channel(L, m, G, slice, qmax);
@@ -973,6 +983,32 @@ squant_model_kernel(const LayerDesc *__restrict__ layers, const Item *__restrict
     } else {
         channel_body<0>(L, m, G, slice, s, mode);
     }
+}
+
+__global__ void __launch_bounds__(kCtaThreads, SQ_MIN_CTAS)
+squant_model_kernel(const __grid_constant__ LaunchTable tbl, int qmax, unsigned mode)
+{
+    extern __shared__ __align__(16) unsigned char smem[];
+    const int item = blockIdx.x;
+    int layer = 0;   // uniform binary search for the last layer whose first item is <= item
+#pragma unroll 1
+    for (int step = 64; step > 0; step >>= 1)
+        if (layer + step < tbl.n_layers && tbl.first_item[layer + step] <= item) layer += step;
+    const LayerDesc &L = tbl.layers[layer];
+    const int ch0 = (item - tbl.first_item[layer]) * (kCtaThreads >> L.g_shift);
+    run_item(L, ch0, smem, qmax, mode);
+}
+
+// The same with the descriptors in a table in global memory (used by the entry point whose
+// table lives in a fixed device array).
+__global__ void __launch_bounds__(kCtaThreads, SQ_MIN_CTAS)
+squant_table_kernel(const LayerDesc *__restrict__ layers, const Item *__restrict__ items, int qmax,
+                    unsigned mode)
+{
+    extern __shared__ __align__(16) unsigned char smem[];
+    const Item it = items[blockIdx.x];
+    const LayerDesc L = layers[it.layer];
+    run_item(L, it.ch0, smem, qmax, mode);
 }
 
 }  // namespace sq
