@@ -169,6 +169,20 @@ int squant_quantize_layer_noalloc(const squant_layer *layer, const squant_option
                                   void *cuda_stream);
 
 /*
+ * Self-check of the arithmetic shortcut in SQuant-E (Algorithm 1 "Scale and SQuant-E").  The 3x3
+ * path does not divide every weight by the channel's scale s; it multiplies by one correctly
+ * rounded reciprocal per channel and corrects the product with two fused multiply-adds, which
+ * yields the correctly rounded quotient.  This call checks that claim on the device: for each of
+ * the n scales (HOST array, each in [2^-60, 2^60], the range in which the shortcut is used) it
+ * runs EVERY fp32 bit pattern w with |w| <= s * qmax through both formulations and counts the
+ * weights whose code or integer perturbation differ.  mismatches (HOST array of n counters) must
+ * come back all zero.  Allocates and frees two small device buffers and waits for the stream.
+ * About 4 ms per scale on a B200.
+ */
+int squant_selfcheck_division(const float *scales, int32_t n, int32_t bits, uint64_t *mismatches,
+                              void *cuda_stream);
+
+/*
  * Waits for all work on the current device and reports whether any kernel of this library gave
  * up one of its bounded waits since the last query (every wait inside the kernels - they only
  * wait for their own asynchronous copies - has an iteration limit, after which the affected

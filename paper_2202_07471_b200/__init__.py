@@ -7,10 +7,10 @@ from .binding import (FLAG_NARROW_RANGE, NOALLOC_MAX_CTAS, MODE_C, MODE_E, MODE_
                       SquantError, alloc_outputs, load_library, squant_device_status, squant_launch_count,
                       squant_plan_info, squant_quantize_layer, squant_quantize_layer_noalloc,
                       squant_quantize_model,
-                      squant_quantize_model_host, squant_shutdown)
+                      squant_quantize_model_host, squant_selfcheck_division, squant_shutdown)
 
 __all__ = ["FLAG_NARROW_RANGE", "NOALLOC_MAX_CTAS", "MODE_C", "MODE_E", "MODE_EKC", "MODE_K", "LayerBuffers",
            "ModelCall", "SquantError", "alloc_outputs", "load_library", "squant_device_status", "squant_launch_count",
            "squant_plan_info", "squant_quantize_layer", "squant_quantize_layer_noalloc",
            "squant_quantize_model",
-           "squant_quantize_model_host", "squant_shutdown"]
+           "squant_quantize_model_host", "squant_selfcheck_division", "squant_shutdown"]

@@ -22,7 +22,7 @@ LIB_PATH = os.path.join(_HERE, "libsquant.so")
 NOALLOC_MAX_CTAS = 32768
 
 EXPORTS = ("squant_quantize_layer", "squant_quantize_layer_noalloc", "squant_quantize_model", "squant_quantize_model_host",
-           "squant_plan_info", "squant_device_status", "squant_launch_count", "squant_strerror", "squant_last_cuda_error",
+           "squant_plan_info", "squant_selfcheck_division", "squant_device_status", "squant_launch_count", "squant_strerror", "squant_last_cuda_error",
            "squant_shutdown")
 
 
@@ -62,8 +62,9 @@ def load_library() -> ctypes.CDLL:
     lib.squant_quantize_model.argtypes = [lp, ctypes.c_int32, op, vp]
     lib.squant_quantize_model_host.argtypes = [lp, ctypes.c_int32, op, vp]
     lib.squant_plan_info.argtypes = [lp, ctypes.c_int32, op, i32p, i32p, i32p]
+    lib.squant_selfcheck_division.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, vp]
     for f in ("squant_quantize_layer", "squant_quantize_layer_noalloc", "squant_quantize_model", "squant_quantize_model_host",
-              "squant_plan_info", "squant_device_status", "squant_shutdown"):
+              "squant_plan_info", "squant_selfcheck_division", "squant_device_status", "squant_shutdown"):
         getattr(lib, f).restype = ctypes.c_int
     lib.squant_launch_count.restype = ctypes.c_int64
     lib.squant_strerror.restype = ctypes.c_char_p
@@ -209,6 +210,17 @@ def squant_plan_info(shapes: Sequence[Sequence[int]], bits: int = 4, mode: int =
     _check(load_library().squant_plan_info(arr, len(shapes), ctypes.byref(opt), ctypes.byref(g),
                                            ctypes.byref(t), ctypes.byref(s)))
     return {"grid_ctas": g.value, "cta_threads": t.value, "dynamic_smem_bytes": s.value}
+
+
+def squant_selfcheck_division(scales, bits: int = 4):
+    """Exhaustive device check of the reciprocal-based division for the given scales (numpy fp32).
+    Returns a numpy uint64 array of mismatch counts (must be all zero)."""
+    import numpy as np
+    sc = np.ascontiguousarray(scales, dtype=np.float32)
+    out = np.zeros(sc.size, dtype=np.uint64)
+    _check(load_library().squant_selfcheck_division(sc.ctypes.data_as(ctypes.c_void_p), sc.size, int(bits),
+                                                   out.ctypes.data_as(ctypes.c_void_p), _stream_handle(None)))
+    return out
 
 
 def squant_device_status() -> None:

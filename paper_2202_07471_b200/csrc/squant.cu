@@ -438,6 +438,35 @@ int squant_plan_info(const squant_layer *layers, int32_t n_layers, const squant_
     return SQUANT_OK;
 }
 
+int squant_selfcheck_division(const float *scales, int32_t n, int32_t bits, uint64_t *mismatches,
+                              void *cuda_stream)
+{
+    if (!scales || !mismatches) return SQUANT_ERR_NULL;
+    if (n <= 0 || n > 65535) return SQUANT_ERR_SHAPE;
+    if (bits < 2 || bits > 8) return SQUANT_ERR_BITS;
+    for (int i = 0; i < n; ++i)
+        if (!(scales[i] >= 0x1p-60f && scales[i] <= 0x1p60f)) return SQUANT_ERR_SHAPE;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    float *d_s = nullptr;
+    unsigned long long *d_m = nullptr;
+    SQ_CUDA(cudaMalloc(&d_s, sizeof(float) * n));
+    cudaError_t e = cudaMalloc(&d_m, sizeof(unsigned long long) * n);
+    if (e != cudaSuccess) { cudaFree(d_s); return cuda_fail(e, "cudaMalloc"); }
+    e = cudaMemcpyAsync(d_s, scales, sizeof(float) * n, cudaMemcpyHostToDevice, stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(d_m, 0, sizeof(unsigned long long) * n, stream);
+    if (e == cudaSuccess) {
+        sq::selfcheck_division_kernel<<<dim3(1184, n), 256, 0, stream>>>(d_s, n, (1 << (bits - 1)) - 1, d_m);
+        e = cudaGetLastError();
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+    }
+    if (e == cudaSuccess) e = cudaMemcpyAsync(mismatches, d_m, sizeof(unsigned long long) * n, cudaMemcpyDeviceToHost, stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+    cudaFree(d_s);
+    cudaFree(d_m);
+    if (e != cudaSuccess) return cuda_fail(e, "squant_selfcheck_division");
+    return SQUANT_OK;
+}
+
 int squant_device_status(void)
 {
     std::lock_guard<std::mutex> lock(g_mutex);

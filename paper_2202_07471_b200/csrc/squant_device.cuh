@@ -954,6 +954,38 @@ __device__ __forceinline__ void channel_body_k9_fast(const LayerDesc &L, int m, 
     }
 }
 
+// ---------------------------------------------------------------- self-check of the fast division
+// For each given scale s (in the fast path's range) and EVERY fp32 bit pattern w with
+// |w| <= s * qmax * (1 + 2^-20) - a superset of what a channel with that scale can contain -
+// compares code and integer perturbation from the reciprocal-based SQuant-E with those from the
+// plain IEEE division.  mismatches[i] counts the disagreements for scales[i].
+__global__ void selfcheck_division_kernel(const float *scales, int n, int qmax,
+                                          unsigned long long *mismatches)
+{
+    const int si = blockIdx.y;
+    if (si >= n) return;
+    const float s = scales[si];
+    const float s2 = __fmul_rn(s, 0x1p-30f);
+    const float y = __frcp_rn(s2);
+    const float lim = __fmul_rn(__fmul_rn(s, static_cast<float>(qmax)), 1.000001f);
+    unsigned long long bad = 0;
+    const unsigned long long total = 1ull << 32;
+    for (unsigned long long b = blockIdx.x * static_cast<unsigned long long>(blockDim.x) + threadIdx.x; b < total;
+         b += static_cast<unsigned long long>(gridDim.x) * blockDim.x) {
+        const float w = __uint_as_float(static_cast<unsigned>(b));
+        if (!(fabsf(w) <= lim)) continue;   // also skips NaN
+        unsigned tb;
+        int Pf_fast;
+        squant_e_fast(w, y, s2, tb, Pf_fast);
+        int q, P;
+        squant_e(w, s, q, P);
+        const int qf = static_cast<int>(static_cast<signed char>(tb & 255u));
+        bad += (qf != q) | (Pf_fast != P);
+    }
+    for (int o = 16; o > 0; o >>= 1) bad += __shfl_xor_sync(kFull, bad, o);
+    if ((threadIdx.x & 31) == 0 && bad) atomicAdd(mismatches + si, bad);
+}
+
 // ---------------------------------------------------------------- grouped launch
 // One CTA per work item.  The descriptor of the CTA's layer comes either from the launch table
 // in the kernel's parameter space (kParams) or from a table in global memory.

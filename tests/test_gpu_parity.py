@@ -152,3 +152,18 @@ def test_repeat_calls_are_deterministic_and_counted():
     torch.cuda.synchronize()
     assert sq.squant_launch_count() == n0 + 2
     assert torch.equal(a.codes, b.codes) and torch.equal(a.kernel_err, b.kernel_err)
+
+
+@pytest.mark.parametrize("bits", [2, 4, 8])
+def test_reciprocal_division_is_exact_for_every_weight(bits):
+    """SQuant-E divides by the channel scale in IEEE fp32 (Algorithm 1, 'Scale and SQuant-E').
+    The 3x3 path replaces the division by a per-channel reciprocal plus two fused corrections;
+    this runs ALL fp32 weights a channel with the given scale can hold through both and wants
+    identical codes and perturbations.  Scales: random ones over the fast range, its two ends,
+    powers of two, all-ones significands (worst case for reciprocals)."""
+    rng = np.random.default_rng(bits)
+    sc = np.exp2(rng.uniform(-60, 60, size=20)).astype(np.float32)
+    special = np.array([2.0 ** -60, 2.0 ** 60, 1.0, 3.0, 1.0 / 3.0, 0.007, 5.9604645e-08], dtype=np.float32)
+    ones = np.array([0x3f7fffff, 0x3fffffff, 0x2b7fffff, 0x5d7fffff, 0x3f800001, 0x3fc00001], dtype=np.uint32).view(np.float32)
+    bad = sq.squant_selfcheck_division(np.concatenate([sc, special, ones]), bits=bits)
+    assert not bad.any(), bad
