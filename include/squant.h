@@ -103,10 +103,11 @@ int squant_quantize_layer(const squant_layer *layer, const squant_options *opt, 
  *   opt               bits / mode / flags shared by all layers; NULL means 4 bit, E|K|C, narrow
  *   cuda_stream       a cudaStream_t (NULL = default stream)
  *
- * The first call with a given (device, descriptors, options) combination builds a launch plan:
- * it allocates a small device table and synchronises the stream once.  Later calls with the
- * same combination only enqueue the kernel.  Outputs are valid when the stream reaches the
- * end of the launch.  All arguments are validated on the host first; a failed call launches
+ * The launch table (layer descriptors) travels by value in the kernel's parameter space: the call
+ * allocates no device memory, uploads nothing and never synchronises; more than 96 layers are
+ * issued as several launches.  Host-side launch tables of recent calls are cached.  Outputs are
+ * valid when the stream reaches the end of the launch.  All arguments are validated on the host
+ * first; a failed call launches
  * nothing and writes nothing.  Returns SQUANT_OK or a negative SQUANT_ERR_* code.
  */
 int squant_quantize_model(const squant_layer *layers, int32_t n_layers, const squant_options *opt,
@@ -136,10 +137,10 @@ int squant_plan_info(const squant_layer *layers, int32_t n_layers, const squant_
  * whose framework has handed every free byte of the GPU to its own memory pool (cudaMalloc then
  * fails or fragments the pool), a latency-critical loop that cannot take the device-wide
  * synchronisation cudaMalloc / cudaFree imply, or a host that is only allowed to run
- * pre-loaded code.  squant_quantize_layer and squant_quantize_model keep their launch table
- * (layer descriptor + one entry per CTA) in cudaMalloc'ed memory; this entry point keeps it in
- * a fixed array that is part of the library image instead, so it calls no cudaMalloc, cudaFree
- * or other allocating routine.  Every GPU that loads the library holds that array
+ * pre-loaded code.  This entry point runs the kernel variant that reads its launch table (layer
+ * descriptor + one entry per CTA) from global memory, and keeps that table in a fixed array
+ * that is part of the library image, so it calls no cudaMalloc, cudaFree or other allocating
+ * routine.  Every GPU that loads the library holds that array
  * (SQUANT_NOALLOC_TABLE_BYTES, about 256 KB) until the process exits.
  *
  *   layer, opt, cuda_stream   as for squant_quantize_layer; DEVICE pointers, caller-owned
