@@ -726,89 +726,26 @@ __device__ __forceinline__ void hist_add(int *hist, int v)
     atomicAdd(&hist[a >> 22], (v > 0 ? 1 : 0) | (v < 0 ? 0x10000 : 0));
 }
 
-__device__ __forceinline__ void channel_body_k9_fast(const LayerDesc &L, int m, const Group &G,
-                                                     unsigned char *slice, float s, unsigned mode)
+// Second half of a fast-path channel: channel sum, SQuant-C by the candidate histogram, flips,
+// patched error sums, stores.  KT = 9: kernel n's candidate byte is cbuf[9 n + vi[n]];
+// KT = 1: every element is its own kernel and candidate (vv = ev = the perturbations, byte n).
+// Needs N % 4 = 0.
+template <int KT>
+__device__ __forceinline__ void finish_channel_hist(const LayerDesc &L, int m, const Group &G,
+                                                    unsigned char *slice, float s, unsigned mode,
+                                                    long long esum, float *kerr)
 {
     const int N = L.N, NK = L.NK;
-    const float *wbuf = reinterpret_cast<const float *>(slice);
     unsigned char *cbuf = slice + L.off_codes;
-    int *ev = reinterpret_cast<int *>(slice + L.off_ev);
-    int *vv = reinterpret_cast<int *>(slice + L.off_vv);
-    unsigned char *vi = slice + L.off_vi;
+    const int *ev = reinterpret_cast<const int *>(slice + L.off_ev);
+    const int *vv = reinterpret_cast<const int *>(slice + L.off_vv);
+    const unsigned char *vi = slice + L.off_vi;
     int *hist = reinterpret_cast<int *>(slice + L.off_hist);
     unsigned char *red = slice + L.off_red;
-    int *bc = reinterpret_cast<int *>(red + 128);               // [0..3] radix-select scratch, [5] list count
+    int *bc = reinterpret_cast<int *>(red + 128);               // [0..3] scan result, [5] list count
     unsigned long long *acc = reinterpret_cast<unsigned long long *>(red + 208);
-    int2 *blist = reinterpret_cast<int2 *>(slice);              // boundary list: reuses the weights' space
-    float *kerr = L.kerr ? L.kerr + static_cast<size_t>(m) * N : nullptr;
-    const bool kvec = (reinterpret_cast<uintptr_t>(kerr) & 15) == 0;
-
-    const float s2 = __fmul_rn(s, 0x1p-30f);
-    const float y = __frcp_rn(s2);
+    int2 *blist = reinterpret_cast<int2 *>(slice + L.off_hist); // boundary list: reuses the histogram after the scan
     const int quads = N >> 2;
-    long long esum = 0;
-    for (int Q = G.t; Q < quads; Q += G.g) {
-        const float4 *src = reinterpret_cast<const float4 *>(wbuf) + Q * 9;
-        unsigned *dst = reinterpret_cast<unsigned *>(cbuf) + Q * 9;
-        float P[36];
-#pragma unroll
-        for (int j = 0; j < 9; ++j) {
-            const float4 w = src[j];
-            unsigned t0, t1, t2, t3;
-            squant_e_fastf(w.x, y, s2, t0, P[4 * j]);
-            squant_e_fastf(w.y, y, s2, t1, P[4 * j + 1]);
-            squant_e_fastf(w.z, y, s2, t2, P[4 * j + 2]);
-            squant_e_fastf(w.w, y, s2, t3, P[4 * j + 3]);
-            dst[j] = __byte_perm(__byte_perm(t0, t1, 0x0040), __byte_perm(t2, t3, 0x0040), 0x5410);
-        }
-        int e4[4], v4[4];
-        unsigned i4 = 0, again = 0;
-        const float *wq = wbuf + Q * 36;
-        unsigned char *cq = cbuf + Q * 36;
-#pragma unroll
-        for (int kq = 0; kq < 4; ++kq) {
-            float Pk[9];
-#pragma unroll
-            for (int i = 0; i < 9; ++i) Pk[i] = P[9 * kq + i];
-            int idx;
-            if (kernel9_fast(Pk, wq + 9 * kq, y, s2, cq + 9 * kq, e4[kq], v4[kq], idx)) {
-                again |= 1u << kq;   // redone exactly below
-                e4[kq] = 0;
-                v4[kq] = 0;
-                idx = 0;
-            }
-            hist_add(hist, v4[kq]);
-            i4 |= static_cast<unsigned>(idx) << (8 * kq);
-        }
-        esum += static_cast<long long>(e4[0] + e4[1]) + (e4[2] + e4[3]);   // pairs fit 32 bits
-        reinterpret_cast<int4 *>(ev)[Q] = make_int4(e4[0], e4[1], e4[2], e4[3]);
-        reinterpret_cast<int4 *>(vv)[Q] = make_int4(v4[0], v4[1], v4[2], v4[3]);
-        reinterpret_cast<unsigned *>(vi)[Q] = i4;
-        if (kerr) {
-            float4 f;
-            f.x = __fmul_rn(__int2float_rn(e4[0]), 0x1p-30f);
-            f.y = __fmul_rn(__int2float_rn(e4[1]), 0x1p-30f);
-            f.z = __fmul_rn(__int2float_rn(e4[2]), 0x1p-30f);
-            f.w = __fmul_rn(__int2float_rn(e4[3]), 0x1p-30f);
-            if (kvec) __stcs(reinterpret_cast<float4 *>(kerr) + Q, f);
-            else { kerr[4 * Q] = f.x; kerr[4 * Q + 1] = f.y; kerr[4 * Q + 2] = f.z; kerr[4 * Q + 3] = f.w; }
-        }
-        if (again) {   // rare: kernels the fast selection handed back
-#pragma unroll 1
-            for (int kq = 0; kq < 4; ++kq) {
-                if (again & (1u << kq)) {
-                    const int n = 4 * Q + kq;
-                    const KernelOut o = kernel9_exact(wbuf + n * 9, y, s2, cbuf + n * 9);
-                    ev[n] = o.e;
-                    vv[n] = o.v;
-                    vi[n] = static_cast<unsigned char>(o.idx);
-                    if (kerr) kerr[n] = __fmul_rn(__int2float_rn(o.e), 0x1p-30f);
-                    hist_add(hist, o.v);
-                    esum += o.e;
-                }
-            }
-        }
-    }
     // channel sum: warp shuffle, then one shared atomic per warp
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) esum += __shfl_xor_sync(kFull, esum, o);
@@ -902,7 +839,7 @@ __device__ __forceinline__ void channel_body_k9_fast(const LayerDesc &L, int m, 
                         }
                     }
                     if (take) {
-                        unsigned char *bp = cbuf + n * 9 + vi[n];
+                        unsigned char *bp = cbuf + (KT == 1 ? n : n * 9 + vi[n]);
                         *bp = static_cast<unsigned char>(*bp - sgn_c);
                         if (kerr) kerr[n] = __fmul_rn(__int2float_rn(ev[n] - sgn_c * kOne), 0x1p-30f);
                     }
@@ -920,7 +857,7 @@ __device__ __forceinline__ void channel_body_k9_fast(const LayerDesc &L, int m, 
                 rank += (o.x > me.x || (o.x == me.x && o.y < me.y)) ? 1 : 0;
             }
             if (rank < rem) {
-                unsigned char *bp = cbuf + me.y * 9 + vi[me.y];
+                unsigned char *bp = cbuf + (KT == 1 ? me.y : me.y * 9 + vi[me.y]);
                 *bp = static_cast<unsigned char>(*bp - sgn_c);
                 if (kerr) kerr[me.y] = __fmul_rn(__int2float_rn(ev[me.y] - sgn_c * kOne), 0x1p-30f);
             }
@@ -952,6 +889,139 @@ __device__ __forceinline__ void channel_body_k9_fast(const LayerDesc &L, int m, 
         L.scales[m] = s;
         if (L.cerr) L.cerr[m] = __fmul_rn(__ll2float_rn(ec), 0x1p-30f);
     }
+}
+
+
+
+__device__ __forceinline__ void channel_body_k9_fast(const LayerDesc &L, int m, const Group &G,
+                                                     unsigned char *slice, float s, unsigned mode)
+{
+    const int N = L.N;
+    const float *wbuf = reinterpret_cast<const float *>(slice);
+    unsigned char *cbuf = slice + L.off_codes;
+    int *ev = reinterpret_cast<int *>(slice + L.off_ev);
+    int *vv = reinterpret_cast<int *>(slice + L.off_vv);
+    unsigned char *vi = slice + L.off_vi;
+    int *hist = reinterpret_cast<int *>(slice + L.off_hist);
+    float *kerr = L.kerr ? L.kerr + static_cast<size_t>(m) * N : nullptr;
+    const bool kvec = (reinterpret_cast<uintptr_t>(kerr) & 15) == 0;
+
+    const float s2 = __fmul_rn(s, 0x1p-30f);
+    const float y = __frcp_rn(s2);
+    const int quads = N >> 2;
+    long long esum = 0;
+    for (int Q = G.t; Q < quads; Q += G.g) {
+        const float4 *src = reinterpret_cast<const float4 *>(wbuf) + Q * 9;
+        unsigned *dst = reinterpret_cast<unsigned *>(cbuf) + Q * 9;
+        float P[36];
+#pragma unroll
+        for (int j = 0; j < 9; ++j) {
+            const float4 w = src[j];
+            unsigned t0, t1, t2, t3;
+            squant_e_fastf(w.x, y, s2, t0, P[4 * j]);
+            squant_e_fastf(w.y, y, s2, t1, P[4 * j + 1]);
+            squant_e_fastf(w.z, y, s2, t2, P[4 * j + 2]);
+            squant_e_fastf(w.w, y, s2, t3, P[4 * j + 3]);
+            dst[j] = __byte_perm(__byte_perm(t0, t1, 0x0040), __byte_perm(t2, t3, 0x0040), 0x5410);
+        }
+        int e4[4], v4[4];
+        unsigned i4 = 0, again = 0;
+        const float *wq = wbuf + Q * 36;
+        unsigned char *cq = cbuf + Q * 36;
+#pragma unroll
+        for (int kq = 0; kq < 4; ++kq) {
+            float Pk[9];
+#pragma unroll
+            for (int i = 0; i < 9; ++i) Pk[i] = P[9 * kq + i];
+            int idx;
+            if (kernel9_fast(Pk, wq + 9 * kq, y, s2, cq + 9 * kq, e4[kq], v4[kq], idx)) {
+                again |= 1u << kq;   // redone exactly below
+                e4[kq] = 0;
+                v4[kq] = 0;
+                idx = 0;
+            }
+            hist_add(hist, v4[kq]);
+            i4 |= static_cast<unsigned>(idx) << (8 * kq);
+        }
+        esum += static_cast<long long>(e4[0] + e4[1]) + (e4[2] + e4[3]);   // pairs fit 32 bits
+        reinterpret_cast<int4 *>(ev)[Q] = make_int4(e4[0], e4[1], e4[2], e4[3]);
+        reinterpret_cast<int4 *>(vv)[Q] = make_int4(v4[0], v4[1], v4[2], v4[3]);
+        reinterpret_cast<unsigned *>(vi)[Q] = i4;
+        if (kerr) {
+            float4 f;
+            f.x = __fmul_rn(__int2float_rn(e4[0]), 0x1p-30f);
+            f.y = __fmul_rn(__int2float_rn(e4[1]), 0x1p-30f);
+            f.z = __fmul_rn(__int2float_rn(e4[2]), 0x1p-30f);
+            f.w = __fmul_rn(__int2float_rn(e4[3]), 0x1p-30f);
+            if (kvec) __stcs(reinterpret_cast<float4 *>(kerr) + Q, f);
+            else { kerr[4 * Q] = f.x; kerr[4 * Q + 1] = f.y; kerr[4 * Q + 2] = f.z; kerr[4 * Q + 3] = f.w; }
+        }
+        if (again) {   // rare: kernels the fast selection handed back
+#pragma unroll 1
+            for (int kq = 0; kq < 4; ++kq) {
+                if (again & (1u << kq)) {
+                    const int n = 4 * Q + kq;
+                    const KernelOut o = kernel9_exact(wbuf + n * 9, y, s2, cbuf + n * 9);
+                    ev[n] = o.e;
+                    vv[n] = o.v;
+                    vi[n] = static_cast<unsigned char>(o.idx);
+                    if (kerr) kerr[n] = __fmul_rn(__int2float_rn(o.e), 0x1p-30f);
+                    hist_add(hist, o.v);
+                    esum += o.e;
+                }
+            }
+        }
+    }
+    finish_channel_hist<9>(L, m, G, slice, s, mode, esum, kerr);
+}
+
+// ---------------------------------------------------------------- channel body, 1x1 fast path
+// Fully connected and pointwise layers (K = 1; needs N % 4 = 0 and 2^-60 <= s <= 2^60).  Every
+// element is its own kernel, SQuant-K is a no-op (Sec. 3.4) and the element's perturbation is its
+// own candidate for SQuant-C.  A thread takes four elements at a time: one 128-bit shared load,
+// the reciprocal-based SQuant-E, one packed word of codes, and the four integer perturbations
+// written back in place of the weights (they are the e' / v arrays of the channel step).
+__device__ __forceinline__ void channel_body_k1_fast(const LayerDesc &L, int m, const Group &G,
+                                                     unsigned char *slice, float s, unsigned mode)
+{
+    const int N = L.N;
+    float4 *wbuf4 = reinterpret_cast<float4 *>(slice);
+    unsigned *cbuf32 = reinterpret_cast<unsigned *>(slice + L.off_codes);
+    int *hist = reinterpret_cast<int *>(slice + L.off_hist);
+    float *kerr = L.kerr ? L.kerr + static_cast<size_t>(m) * N : nullptr;
+    const bool kvec = (reinterpret_cast<uintptr_t>(kerr) & 15) == 0;
+    const float s2 = __fmul_rn(s, 0x1p-30f);
+    const float y = __frcp_rn(s2);
+    const int quads = N >> 2;
+    long long esum = 0;
+    for (int Q = G.t; Q < quads; Q += G.g) {
+        const float4 w = wbuf4[Q];
+        unsigned t0, t1, t2, t3;
+        int4 P;
+        squant_e_fast(w.x, y, s2, t0, P.x);
+        squant_e_fast(w.y, y, s2, t1, P.y);
+        squant_e_fast(w.z, y, s2, t2, P.z);
+        squant_e_fast(w.w, y, s2, t3, P.w);
+        cbuf32[Q] = __byte_perm(__byte_perm(t0, t1, 0x0040), __byte_perm(t2, t3, 0x0040), 0x5410);
+        reinterpret_cast<int4 *>(wbuf4)[Q] = P;
+        if (mode & 4u) {
+            hist_add(hist, P.x);
+            hist_add(hist, P.y);
+            hist_add(hist, P.z);
+            hist_add(hist, P.w);
+        }
+        esum += static_cast<long long>(P.x + P.y) + (P.z + P.w);   // pairs fit 32 bits
+        if (kerr) {
+            float4 f;
+            f.x = __fmul_rn(__int2float_rn(P.x), 0x1p-30f);
+            f.y = __fmul_rn(__int2float_rn(P.y), 0x1p-30f);
+            f.z = __fmul_rn(__int2float_rn(P.z), 0x1p-30f);
+            f.w = __fmul_rn(__int2float_rn(P.w), 0x1p-30f);
+            if (kvec) __stcs(reinterpret_cast<float4 *>(kerr) + Q, f);
+            else { kerr[4 * Q] = f.x; kerr[4 * Q + 1] = f.y; kerr[4 * Q + 2] = f.z; kerr[4 * Q + 3] = f.w; }
+        }
+    }
+    finish_channel_hist<1>(L, m, G, slice, s, mode, esum, kerr);
 }
 
 // ---------------------------------------------------------------- self-check of the fast division
@@ -1006,7 +1076,10 @@ __device__ __forceinline__ void run_item(const LayerDesc &L, int ch0, unsigned c
     const float s = stage_channel(L, m, G, slice, qmax);
     if (s == 0.0f) return;   // staging wait ran out (status word set); nothing is written
     if (L.K == 1) {
-        channel_body<1>(L, m, G, slice, s, mode);
+        if ((L.N & 3) == 0 && s >= 0x1p-60f && s <= 0x1p60f)
+            channel_body_k1_fast(L, m, G, slice, s, mode);
+        else
+            channel_body<1>(L, m, G, slice, s, mode);
     } else if (L.K == 9) {
         if ((L.N & 3) == 0 && (mode & 2u) && s >= 0x1p-60f && s <= 0x1p60f)
             channel_body_k9_fast(L, m, G, slice, s, mode);
