@@ -167,3 +167,31 @@ def test_reciprocal_division_is_exact_for_every_weight(bits):
     ones = np.array([0x3f7fffff, 0x3fffffff, 0x2b7fffff, 0x5d7fffff, 0x3f800001, 0x3fc00001], dtype=np.uint32).view(np.float32)
     bad = sq.squant_selfcheck_division(np.concatenate([sc, special, ones]), bits=bits)
     assert not bad.any(), bad
+
+
+def test_more_layers_than_one_launch_table_holds():
+    """More than 96 layers are issued as several launches; results do not depend on the split."""
+    shapes = [(3 + (i % 5), 8 + 4 * (i % 7), 3, 3) if i % 3 else (5, 16 + 4 * (i % 9), 1, 1) for i in range(205)]
+    ws = [W.random_layer(s, seed=1000 + i) for i, s in enumerate(shapes)]
+    n0 = sq.squant_launch_count()
+    bufs = run_gpu(ws, 4, EKC)
+    assert sq.squant_launch_count() == n0 + 3
+    for i, (b, w) in enumerate(zip(bufs, ws)):
+        assert_layer_equal(b, w, 4, EKC, tag=f"layer {i} {shapes[i]}")
+
+
+def test_non_finite_inputs_do_not_disturb_other_channels():
+    """NaN / Inf weights are outside the method's domain; their channels produce unspecified
+    codes, but every index the kernel forms stays in bounds and finite channels are unaffected."""
+    for shape in [(8, 64, 3, 3), (8, 256, 1, 1), (8, 10, 5, 5), (8, 2048, 3, 3)]:
+        w = W.random_layer(shape, seed=77)
+        bad = w.copy()
+        bad[1].reshape(-1)[3] = np.nan
+        bad[2].reshape(-1)[5] = np.inf
+        bad[3].reshape(-1)[::7] = -np.inf
+        bad[5].reshape(-1)[:] = np.nan
+        (b,) = run_gpu([bad], 4, EKC)
+        r = oracle.quantize_layer(w, bits=4, mode=EKC)
+        for c in (0, 4, *range(6, shape[0])):
+            assert np.array_equal(b.codes[c].cpu().numpy(), r.codes[c])
+            assert b.scales[c].item() == r.scales[c]
