@@ -50,6 +50,9 @@ extern "C" {
 /* flags */
 #define SQUANT_FLAG_NARROW_RANGE 1u /* codes in [-qmax, qmax] (default); without it the lower
                                        bound is -qmax-1, which the absmax scale never reaches */
+#define SQUANT_FLAG_PACK_INT4 2u    /* bits <= 4 only: codes are emitted two per byte (two's
+                                       complement nibbles, low nibble = even flat index), every
+                                       output channel in a row of ceil(cin*kh*kw / 2) bytes */
 
 /* error codes (0 = success) */
 #define SQUANT_OK 0
@@ -82,7 +85,8 @@ typedef struct squant_layer {
     const float *w;      /* in : [cout][cin][kh][kw] fp32, finite values, 4-byte aligned
                                  (16-byte alignment of every channel enables the fast loads) */
     int32_t cout, cin, kh, kw;
-    int8_t *codes;       /* out: [cout][cin][kh][kw] int8 */
+    int8_t *codes;       /* out: [cout][cin][kh][kw] int8, or with SQUANT_FLAG_PACK_INT4
+                                 [cout][ceil(cin*kh*kw / 2)] bytes of nibble pairs */
     float *scales;       /* out: [cout] */
     float *kernel_err;   /* out, may be NULL: [cout][cin] final signed sum of a kernel's
                                  perturbations, (float)(integer sum) * 2^-30 */

@@ -17,6 +17,7 @@ from . import build as _build
 MODE_E, MODE_K, MODE_C = 1, 2, 4
 MODE_EKC = MODE_E | MODE_K | MODE_C
 FLAG_NARROW_RANGE = 1
+FLAG_PACK_INT4 = 2
 ONE = 1 << 30
 HALF = 1 << 29
 
@@ -43,7 +44,7 @@ def _load():
 
 @dataclass
 class OracleResult:
-    codes: np.ndarray                      # int8, shape of the weights
+    codes: np.ndarray                      # int8, shape of the weights ([M, ceil(N*K/2)] if packed)
     scales: np.ndarray                     # fp32 [M]
     kernel_err: np.ndarray                 # fp32 [M, N]
     channel_err: np.ndarray                # fp32 [M]
@@ -59,7 +60,10 @@ def quantize_layer(w: np.ndarray, bits: int = 4, mode: int = MODE_EKC,
         raise ValueError("weights need at least [M, N]")
     M, N = int(w.shape[0]), int(w.shape[1])
     K = int(np.prod(w.shape[2:])) if w.ndim > 2 else 1
-    codes = np.empty(w.shape, dtype=np.int8)
+    if flags & FLAG_PACK_INT4:
+        codes = np.empty((M, (N * K + 1) // 2), dtype=np.int8)
+    else:
+        codes = np.empty(w.shape, dtype=np.int8)
     scales = np.empty(M, dtype=np.float32)
     kerr = np.empty((M, N), dtype=np.float32)
     cerr = np.empty(M, dtype=np.float32)

@@ -60,13 +60,15 @@
 #define SQO_HALF ((int64_t)1 << 29)
 
 enum { SQO_MODE_E = 1u, SQO_MODE_K = 2u, SQO_MODE_C = 4u };
-enum { SQO_FLAG_NARROW_RANGE = 1u };
+enum { SQO_FLAG_NARROW_RANGE = 1u, SQO_FLAG_PACK_INT4 = 2u };
 enum { SQO_OK = 0, SQO_ERR_ARG = -1, SQO_ERR_NOMEM = -2 };
 
 typedef struct {
     int32_t bits;    /* 2..8 */
     uint32_t mode;   /* SQO_MODE_E | SQO_MODE_K | SQO_MODE_C */
-    uint32_t flags;  /* SQO_FLAG_NARROW_RANGE: codes in [-qmax, qmax] */
+    uint32_t flags;  /* SQO_FLAG_NARROW_RANGE: codes in [-qmax, qmax];
+                        SQO_FLAG_PACK_INT4 (bits <= 4): two codes per byte, low nibble = even flat
+                        index, ceil(N*K/2) bytes per output channel */
 } sqo_options;
 
 typedef struct {
@@ -217,13 +219,21 @@ static void sqo_channel(const float *w, int32_t N, int32_t K, const sqo_options 
         if (kernel_err) kernel_err[n] = (float)e * 0x1p-30f;
     }
     if (channel_err) *channel_err = (float)total * 0x1p-30f;
-    for (int32_t j = 0; j < NK; ++j) codes[j] = (int8_t)q[j];
+    if (opt->flags & SQO_FLAG_PACK_INT4) {
+        for (int32_t j = 0; j < NK; j += 2) {
+            unsigned lo = (unsigned)q[j] & 15u;
+            unsigned hi = (j + 1 < NK) ? ((unsigned)q[j + 1] & 15u) : 0u;
+            codes[j / 2] = (int8_t)(lo | (hi << 4));
+        }
+    } else {
+        for (int32_t j = 0; j < NK; ++j) codes[j] = (int8_t)q[j];
+    }
 }
 
 /*
  * Quantize one layer.  All pointers are HOST pointers owned by the caller.
  *   w            [M][N][K] fp32
- *   codes        out [M][N][K] int8
+ *   codes        out [M][N][K] int8 (with SQO_FLAG_PACK_INT4: [M][ceil(N*K/2)] nibble pairs)
  *   scales       out [M]
  *   kernel_err   out [M][N], may be NULL
  *   channel_err  out [M], may be NULL
@@ -237,6 +247,7 @@ int sqo_quantize_layer(const float *w, int32_t M, int32_t N, int32_t K, const sq
 {
     if (!w || !opt || !codes || !scales || M < 0 || N <= 0 || K <= 0) return SQO_ERR_ARG;
     if (opt->bits < 2 || opt->bits > 8 || !(opt->mode & SQO_MODE_E)) return SQO_ERR_ARG;
+    if ((opt->flags & SQO_FLAG_PACK_INT4) && opt->bits > 4) return SQO_ERR_ARG;
     if ((int64_t)N * K > (int64_t)1 << 30) return SQO_ERR_ARG;
     const size_t NK = (size_t)N * K;
     sqo_work wk;
@@ -251,7 +262,8 @@ int sqo_quantize_layer(const float *w, int32_t M, int32_t N, int32_t K, const sq
         rc = SQO_ERR_NOMEM;
     } else {
         for (int32_t m = 0; m < M; ++m) {
-            sqo_channel(w + (size_t)m * NK, N, K, opt, &wk, codes + (size_t)m * NK, scales + m,
+            sqo_channel(w + (size_t)m * NK, N, K, opt, &wk,
+                        codes + (size_t)m * ((opt->flags & SQO_FLAG_PACK_INT4) ? (NK + 1) / 2 : NK), scales + m,
                         kernel_err ? kernel_err + (size_t)m * N : NULL,
                         channel_err ? channel_err + m : NULL);
             if (pert) memcpy(pert + (size_t)m * NK, wk.P, NK * sizeof(int32_t));

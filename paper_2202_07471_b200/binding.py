@@ -15,6 +15,7 @@ import torch
 MODE_E, MODE_K, MODE_C = 1, 2, 4
 MODE_EKC = MODE_E | MODE_K | MODE_C
 FLAG_NARROW_RANGE = 1
+FLAG_PACK_INT4 = 2
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libsquant.so")
@@ -93,16 +94,18 @@ class LayerBuffers:
 
 
 def alloc_outputs(w: torch.Tensor, kernel_err: bool = True, channel_err: bool = True,
-                  pin: bool = False) -> LayerBuffers:
-    """Allocate output tensors next to `w` ([cout, cin, kh, kw], [cout, cin, k] or [cout, cin])."""
+                  pin: bool = False, pack_int4: bool = False) -> LayerBuffers:
+    """Allocate output tensors next to `w` ([cout, cin, kh, kw], [cout, cin, k] or [cout, cin]).
+    With pack_int4 the codes tensor is [cout, ceil(cin*kh*kw / 2)] (for FLAG_PACK_INT4)."""
     if w.dtype != torch.float32 or not w.is_contiguous() or w.dim() < 2:
         raise ValueError("weights must be a contiguous fp32 tensor [cout, cin, ...]")
     kw = dict(device=w.device)
     if pin and not w.is_cuda:
         kw["pin_memory"] = True
     m, n = w.shape[0], w.shape[1]
+    cshape = (m, (w[0].numel() + 1) // 2) if pack_int4 else w.shape
     return LayerBuffers(
-        w, torch.empty(w.shape, dtype=torch.int8, **kw), torch.empty(m, dtype=torch.float32, **kw),
+        w, torch.empty(cshape, dtype=torch.int8, **kw), torch.empty(m, dtype=torch.float32, **kw),
         torch.empty((m, n), dtype=torch.float32, **kw) if kernel_err else None,
         torch.empty(m, dtype=torch.float32, **kw) if channel_err else None)
 

@@ -74,7 +74,8 @@ int validate(const squant_layer *layers, int32_t n_layers, const squant_options 
     if (n_layers > 0 && !layers) return SQUANT_ERR_NULL;
     if (o.bits < 2 || o.bits > 8) return SQUANT_ERR_BITS;
     if (!(o.mode & SQUANT_MODE_E) || (o.mode & ~SQUANT_MODE_EKC)) return SQUANT_ERR_MODE;
-    if (o.flags & ~SQUANT_FLAG_NARROW_RANGE) return SQUANT_ERR_MODE;
+    if (o.flags & ~(SQUANT_FLAG_NARROW_RANGE | SQUANT_FLAG_PACK_INT4)) return SQUANT_ERR_MODE;
+    if ((o.flags & SQUANT_FLAG_PACK_INT4) && o.bits > 4) return SQUANT_ERR_BITS;
     for (int i = 0; i < n_layers; ++i) {
         const squant_layer &l = layers[i];
         if (l.cout <= 0 || l.cin <= 0 || l.kh <= 0 || l.kw <= 0) return SQUANT_ERR_SHAPE;
@@ -126,7 +127,7 @@ int build_plan(const squant_layer *layers, int32_t n_layers, const squant_option
                HostPlan &p)
 {
     p.qmax = (1 << (o.bits - 1)) - 1;
-    p.mode = o.mode;
+    p.mode = o.mode | ((o.flags & SQUANT_FLAG_PACK_INT4) ? sq::kModePackInt4 : 0u);
     p.layers.resize(n_layers);
     p.smem_bytes = 0;
     struct Batch { int64_t work; int layer; int ch0; };
@@ -164,7 +165,7 @@ int build_param_plan(const squant_layer *layers, int32_t n_layers, const squant_
                      int max_smem, ParamPlan &p)
 {
     p.qmax = (1 << (o.bits - 1)) - 1;
-    p.mode = o.mode;
+    p.mode = o.mode | ((o.flags & SQUANT_FLAG_PACK_INT4) ? sq::kModePackInt4 : 0u);
     p.smem_bytes = 0;
     std::vector<LayerDesc> descs(n_layers);
     std::vector<int> order(n_layers);
@@ -343,7 +344,9 @@ int squant_quantize_model_host(const squant_layer *layers, int32_t n_layers,
         const squant_layer &l = layers[i];
         const size_t n = static_cast<size_t>(l.cin) * l.kh * l.kw * l.cout;
         off[5 * i + 0] = total; total += align256(n * 4);
-        off[5 * i + 1] = total; total += align256(n);
+        const size_t code_bytes = (o.flags & SQUANT_FLAG_PACK_INT4)
+                                      ? static_cast<size_t>(l.cout) * ((static_cast<size_t>(l.cin) * l.kh * l.kw + 1) / 2) : n;
+        off[5 * i + 1] = total; total += align256(code_bytes);
         off[5 * i + 2] = total; total += align256(static_cast<size_t>(l.cout) * 4);
         off[5 * i + 3] = total; total += l.kernel_err ? align256(static_cast<size_t>(l.cout) * l.cin * 4) : 0;
         off[5 * i + 4] = total; total += l.channel_err ? align256(static_cast<size_t>(l.cout) * 4) : 0;
@@ -375,7 +378,9 @@ int squant_quantize_model_host(const squant_layer *layers, int32_t n_layers,
     for (int i = 0; i < n_layers; ++i) {
         const squant_layer &l = layers[i];
         const size_t n = static_cast<size_t>(l.cin) * l.kh * l.kw * l.cout;
-        SQ_CUDA(cudaMemcpyAsync(l.codes, dev[i].codes, n, cudaMemcpyDeviceToHost, stream));
+        const size_t code_bytes = (o.flags & SQUANT_FLAG_PACK_INT4)
+                                      ? static_cast<size_t>(l.cout) * ((static_cast<size_t>(l.cin) * l.kh * l.kw + 1) / 2) : n;
+        SQ_CUDA(cudaMemcpyAsync(l.codes, dev[i].codes, code_bytes, cudaMemcpyDeviceToHost, stream));
         SQ_CUDA(cudaMemcpyAsync(l.scales, dev[i].scales, static_cast<size_t>(l.cout) * 4, cudaMemcpyDeviceToHost, stream));
         if (l.kernel_err)
             SQ_CUDA(cudaMemcpyAsync(l.kernel_err, dev[i].kernel_err, static_cast<size_t>(l.cout) * l.cin * 4, cudaMemcpyDeviceToHost, stream));
@@ -487,7 +492,7 @@ const char *squant_strerror(int code)
         case SQUANT_OK: return "success";
         case SQUANT_ERR_NULL: return "a required pointer is NULL";
         case SQUANT_ERR_SHAPE: return "a layer dimension is not positive or the element count overflows";
-        case SQUANT_ERR_BITS: return "bits must be in 2..8";
+        case SQUANT_ERR_BITS: return "bits must be in 2..8 (2..4 with SQUANT_FLAG_PACK_INT4)";
         case SQUANT_ERR_MODE: return "mode mask must contain E and be one of E, E|K, E|K|C (E|C only for 1x1 kernels); unknown flag bits are rejected";
         case SQUANT_ERR_ALIGN: return "float pointers must be 4-byte aligned";
         case SQUANT_ERR_TOO_WIDE: return "an output channel (cin*kh*kw) does not fit the on-chip path";

@@ -621,13 +621,55 @@ __device__ __forceinline__ ChannelStep channel_step(const LayerDesc &L, const Gr
     return c;
 }
 
+// ---------------------------------------------------------------- emit one channel
+// Codes of one channel from the staging buffer to global memory, then scale and channel error.
+// Called by the whole group right after a group barrier that made the final staged codes
+// visible.  int8: N*K bytes; packed int4 (kModePackInt4 in `mode`, bits <= 4): two codes per byte,
+// low nibble = even flat index, ceil(N*K / 2) bytes per output channel, packed into `scratch`
+// (shared memory that is dead by now) first.  Aligned rows leave by one bulk asynchronous copy.
+constexpr unsigned kModePackInt4 = 0x100u;
+
+__device__ __forceinline__ void emit_channel(const LayerDesc &L, int m, const Group &G,
+                                             const unsigned char *cbuf, unsigned char *scratch, float s,
+                                             long long ec, unsigned mode)
+{
+    const int NK = L.NK;
+    const unsigned char *src = cbuf;
+    int row = NK;
+    if (mode & kModePackInt4) {
+        row = (NK + 1) >> 1;
+        const int pairs = NK >> 1;
+        for (int i = G.t; i < pairs; i += G.g)
+            scratch[i] = static_cast<unsigned char>((cbuf[2 * i] & 15) | (cbuf[2 * i + 1] << 4));
+        if ((NK & 1) && G.t == 0) scratch[pairs] = static_cast<unsigned char>(cbuf[NK - 1] & 15);
+        G.sync();
+        src = scratch;
+    }
+    unsigned char *cg = reinterpret_cast<unsigned char *>(L.codes) + static_cast<size_t>(m) * row;
+    const bool aligned = (reinterpret_cast<uintptr_t>(cg) & 15) == 0;
+    if (aligned && (row & 15) == 0) {
+        if (G.t == 0) bulk_store(cg, src, static_cast<unsigned>(row));
+    } else if (aligned) {
+        const int nv = row >> 4;
+        for (int i = G.t; i < nv; i += G.g) __stcs(reinterpret_cast<int4 *>(cg) + i, reinterpret_cast<const int4 *>(src)[i]);
+        for (int i = (nv << 4) + G.t; i < row; i += G.g) cg[i] = src[i];
+    } else {
+        for (int i = G.t; i < row; i += G.g) cg[i] = src[i];
+    }
+    if (G.t == 0) {
+        L.scales[m] = s;
+        if (L.cerr) L.cerr[m] = __fmul_rn(__ll2float_rn(ec), 0x1p-30f);
+        bulk_store_wait();   // shared memory must stay intact until the bulk copy has read it
+    }
+}
+
 // ---------------------------------------------------------------- channel body, any kernel size
 template <int KT>
 __device__ __forceinline__ void channel_body(const LayerDesc &L, int m, const Group &G,
                                              unsigned char *slice, float s, unsigned mode)
 {
     const int K = KT ? KT : L.K;
-    const int N = L.N, NK = L.NK;
+    const int N = L.N;
     float *wbuf = reinterpret_cast<float *>(slice);
     int8_t *cbuf = reinterpret_cast<int8_t *>(slice + L.off_codes);
     int *ev = reinterpret_cast<int *>(slice + L.off_ev);
@@ -687,21 +729,8 @@ __device__ __forceinline__ void channel_body(const LayerDesc &L, int m, const Gr
     }
     G.sync();
 
-    // ---- codes, scale, channel error
-    int8_t *cg = L.codes + static_cast<size_t>(m) * NK;
-    if ((reinterpret_cast<uintptr_t>(cg) & 15) == 0) {
-        const int nv = NK >> 4;
-        const int4 *src = reinterpret_cast<const int4 *>(cbuf);
-        int4 *dst = reinterpret_cast<int4 *>(cg);
-        for (int i = G.t; i < nv; i += G.g) __stcs(dst + i, src[i]);
-        for (int i = (nv << 4) + G.t; i < NK; i += G.g) cg[i] = cbuf[i];
-    } else {
-        for (int i = G.t; i < NK; i += G.g) cg[i] = cbuf[i];
-    }
-    if (G.t == 0) {
-        L.scales[m] = s;
-        if (L.cerr) L.cerr[m] = __fmul_rn(__ll2float_rn(ec), 0x1p-30f);
-    }
+    // ---- codes, scale, channel error (the staged weights / perturbations are dead: scratch)
+    emit_channel(L, m, G, reinterpret_cast<const unsigned char *>(cbuf), slice, s, ec, mode);
 }
 
 // ---------------------------------------------------------------- channel body, 3x3 fast path
@@ -735,7 +764,7 @@ __device__ __forceinline__ void finish_channel_hist(const LayerDesc &L, int m, c
                                                     unsigned char *slice, float s, unsigned mode,
                                                     long long esum, float *kerr)
 {
-    const int N = L.N, NK = L.NK;
+    const int N = L.N;
     unsigned char *cbuf = slice + L.off_codes;
     const int *ev = reinterpret_cast<const int *>(slice + L.off_ev);
     const int *vv = reinterpret_cast<const int *>(slice + L.off_vv);
@@ -865,30 +894,8 @@ __device__ __forceinline__ void finish_channel_hist(const LayerDesc &L, int m, c
         G.sync();
     }
 
-    // ---- codes, scale, channel error
-    int8_t *cg = L.codes + static_cast<size_t>(m) * NK;
-    if ((reinterpret_cast<uintptr_t>(cg) & 15) == 0 && (NK & 15) == 0) {
-        if (G.t == 0) {   // one bulk asynchronous copy of the staged codes
-            bulk_store(cg, cbuf, static_cast<unsigned>(NK));
-            L.scales[m] = s;
-            if (L.cerr) L.cerr[m] = __fmul_rn(__ll2float_rn(ec), 0x1p-30f);
-            bulk_store_wait();   // shared memory must stay intact until it has been read
-        }
-        return;
-    }
-    if ((reinterpret_cast<uintptr_t>(cg) & 15) == 0) {
-        const int nv = NK >> 4;
-        const int4 *src = reinterpret_cast<const int4 *>(cbuf);
-        int4 *dst = reinterpret_cast<int4 *>(cg);
-        for (int i = G.t; i < nv; i += G.g) __stcs(dst + i, src[i]);
-        for (int i = (nv << 4) + G.t; i < NK; i += G.g) cg[i] = static_cast<int8_t>(cbuf[i]);
-    } else {
-        for (int i = G.t; i < NK; i += G.g) cg[i] = static_cast<int8_t>(cbuf[i]);
-    }
-    if (G.t == 0) {
-        L.scales[m] = s;
-        if (L.cerr) L.cerr[m] = __fmul_rn(__ll2float_rn(ec), 0x1p-30f);
-    }
+    // ---- codes, scale, channel error (the staged weights / perturbations are dead: scratch)
+    emit_channel(L, m, G, cbuf, slice, s, ec, mode);
 }
 
 

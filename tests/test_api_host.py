@@ -51,6 +51,7 @@ def test_plan_geometry_for_the_five_configs():
     ((4, 3, 3, 3), {"bits": 1}, -3), ((4, 3, 3, 3), {"bits": 9}, -3),
     ((4, 3, 3, 3), {"mode": 2}, -4), ((4, 3, 3, 3), {"mode": 8 | 1}, -4),
     ((4, 3, 3, 3), {"mode": 1 | 4}, -4), ((4, 3, 3, 3), {"flags": 16}, -4),
+    ((4, 3, 3, 3), {"bits": 6, "flags": 3}, -3),
     ((4, 70000, 1, 1), {}, -6), ((4, 8000, 3, 3), {}, -6),
 ])
 def test_invalid_arguments_are_rejected(shape, kw, code):

@@ -195,3 +195,24 @@ def test_non_finite_inputs_do_not_disturb_other_channels():
         for c in (0, 4, *range(6, shape[0])):
             assert np.array_equal(b.codes[c].cpu().numpy(), r.codes[c])
             assert b.scales[c].item() == r.scales[c]
+
+
+@pytest.mark.parametrize("bits", [3, 4])
+def test_packed_int4_output(bits):
+    """SQUANT_FLAG_PACK_INT4: nibble pairs, rows of ceil(NK/2) bytes; all kernel paths, odd and
+    even row lengths, bulk-store and plain-store rows."""
+    shapes = [(6, 64, 3, 3), (3, 2048, 3, 3), (5, 256, 1, 1), (7, 33, 1, 1), (4, 3, 5, 5), (9, 1, 3, 3), (3, 7, 3, 3)]
+    ws = [adversarial_layer(s, seed=3 * bits + i) for i, s in enumerate(shapes)]
+    flags = sq.FLAG_NARROW_RANGE | sq.FLAG_PACK_INT4
+    bufs = [sq.alloc_outputs(torch.from_numpy(w).cuda(), pack_int4=True) for w in ws]
+    for b in bufs:
+        b.codes.fill_(-128)
+    sq.squant_quantize_model(bufs, bits=bits, mode=EKC, flags=flags)
+    sq.squant_device_status()
+    for b, w, shp in zip(bufs, ws, shapes):
+        r = oracle.quantize_layer(w, bits=bits, mode=EKC, flags=flags)
+        assert np.array_equal(b.codes.cpu().numpy(), r.codes), f"shape {shp}"
+        assert np.array_equal(b.scales.cpu().numpy(), r.scales)
+        assert np.array_equal(b.kernel_err.cpu().numpy(), r.kernel_err)
+    with pytest.raises(sq.SquantError):
+        sq.squant_quantize_model(bufs[:1], bits=8, flags=flags)

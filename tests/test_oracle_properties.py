@@ -380,3 +380,30 @@ def test_range_exclusion_binds_only_on_a_very_wide_kernel():
     assert r.codes[0, 0, 0] == 127                  # the edge element stayed
     assert r.codes[0, 0, 1] == 1 and int(r.codes[0, 0, 2:].max()) == 0
     assert abs(float(r.kernel_err[0, 0])) <= 0.5
+
+
+def _unpack_int4(packed, nk):
+    u = packed.astype(np.uint8)
+    out = np.empty((packed.shape[0], 2 * packed.shape[1]), dtype=np.int16)
+    out[:, 0::2] = u & 15
+    out[:, 1::2] = u >> 4
+    out = np.where(out > 7, out - 16, out)
+    return out[:, :nk].astype(np.int8)
+
+
+@pytest.mark.parametrize("bits", [2, 3, 4])
+@pytest.mark.parametrize("shape", [(5, 7, 3, 3), (4, 33, 1, 1), (3, 2, 5, 5), (2, 1, 3, 3)])
+def test_packed_int4_output_is_a_relabelling(shape, bits):
+    """Packed output: two's-complement nibbles, low nibble = even flat index, rows of ceil(NK/2)
+    bytes; unpacking gives exactly the int8 codes, everything else is unchanged."""
+    w = _layer(shape, seed=bits)
+    a = oracle.quantize_layer(w, bits=bits, mode=EKC)
+    b = oracle.quantize_layer(w, bits=bits, mode=EKC, flags=oracle.FLAG_NARROW_RANGE | oracle.FLAG_PACK_INT4)
+    nk = int(np.prod(shape[1:]))
+    assert b.codes.shape == (shape[0], (nk + 1) // 2)
+    assert np.array_equal(_unpack_int4(b.codes, nk), a.codes.reshape(shape[0], -1))
+    assert np.array_equal(a.scales, b.scales) and np.array_equal(a.kernel_err, b.kernel_err)
+    if nk & 1:
+        assert not ((b.codes[:, -1].astype(np.uint8) >> 4).any())   # pad nibble is zero
+    with pytest.raises(ValueError):
+        oracle.quantize_layer(w, bits=6, flags=oracle.FLAG_PACK_INT4)
