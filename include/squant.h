@@ -41,7 +41,9 @@
 extern "C" {
 #endif
 
-/* stages to run (bit mask); SQUANT_MODE_E is mandatory */
+/* stages to run (bit mask); SQUANT_MODE_E is mandatory.  E, E|K, E|C and E|K|C are the four
+ * variants of the paper's granularity ablation (Table 5); without SQUANT_MODE_K every element
+ * is its own candidate for SQuant-C. */
 #define SQUANT_MODE_E 1u
 #define SQUANT_MODE_K 2u
 #define SQUANT_MODE_C 4u
@@ -59,8 +61,7 @@ extern "C" {
 #define SQUANT_ERR_NULL (-1)        /* a required pointer is NULL */
 #define SQUANT_ERR_SHAPE (-2)       /* a dimension is <= 0 or the element count overflows */
 #define SQUANT_ERR_BITS (-3)        /* bits outside 2..8 */
-#define SQUANT_ERR_MODE (-4)        /* mode mask without SQUANT_MODE_E, unknown bits, or a
-                                       combination that is not built (E|C on kernels > 1x1) */
+#define SQUANT_ERR_MODE (-4)        /* mode mask without SQUANT_MODE_E, or unknown mode / flag bits */
 #define SQUANT_ERR_ALIGN (-5)       /* weights / scales / error pointers not 4-byte aligned */
 #define SQUANT_ERR_TOO_WIDE (-6)    /* one output channel does not fit the on-chip path */
 #define SQUANT_ERR_CUDA (-7)        /* a CUDA runtime call failed; see squant_last_cuda_error() */

@@ -84,9 +84,6 @@ int validate(const squant_layer *layers, int32_t n_layers, const squant_options 
         if (k > 65535 || nk > (1ll << 30)) return SQUANT_ERR_SHAPE;
         if (static_cast<int64_t>(l.cout) * nk > (1ll << 40)) return SQUANT_ERR_SHAPE;
         if (nk > kMaxChannelElems) return SQUANT_ERR_TOO_WIDE;
-        // E|C without K on kernels larger than 1x1 makes every element a channel candidate;
-        // that selection is not built.
-        if ((o.mode & SQUANT_MODE_C) && !(o.mode & SQUANT_MODE_K) && k > 1) return SQUANT_ERR_MODE;
         if (need_pointers) {
             if (!l.w || !l.codes || !l.scales) return SQUANT_ERR_NULL;
             if ((reinterpret_cast<uintptr_t>(l.w) & 3) || (reinterpret_cast<uintptr_t>(l.scales) & 3) ||
@@ -100,7 +97,7 @@ int validate(const squant_layer *layers, int32_t n_layers, const squant_options 
 
 // Device-side descriptor of one layer: group size and the layout of a group's shared-memory
 // slice.  Returns the dynamic shared memory one CTA needs for this layer.
-int64_t layout_layer(const squant_layer &l, LayerDesc &d)
+int64_t layout_layer(const squant_layer &l, LayerDesc &d, unsigned mode)
 {
     d.w = l.w; d.codes = l.codes; d.scales = l.scales; d.kerr = l.kernel_err; d.cerr = l.channel_err;
     d.M = l.cout; d.N = l.cin; d.K = l.kh * l.kw; d.NK = d.N * d.K;
@@ -109,7 +106,8 @@ int64_t layout_layer(const squant_layer &l, LayerDesc &d)
     while ((1 << d.g_shift) < d.g) ++d.g_shift;
     int off = align16(4 * d.NK);              // staged weights
     d.off_codes = off; off += align16(d.NK);  // staged codes
-    if (d.K == 1) {                           // 1x1: perturbations overwrite the weights
+    const bool ec_only = (mode & SQUANT_MODE_C) && !(mode & SQUANT_MODE_K);   // elements are the candidates
+    if (d.K == 1 || ec_only) {                // perturbations overwrite the weights
         d.off_ev = 0; d.off_vv = 0; d.off_vi = 0;
     } else {
         d.off_ev = off; off += align16(4 * d.N);
@@ -134,7 +132,7 @@ int build_plan(const squant_layer *layers, int32_t n_layers, const squant_option
     std::vector<Batch> batches;
     for (int i = 0; i < n_layers; ++i) {
         LayerDesc &d = p.layers[i];
-        const int64_t cta_smem = layout_layer(layers[i], d);
+        const int64_t cta_smem = layout_layer(layers[i], d, o.mode);
         const int groups = sq::kCtaThreads / d.g;
         if (cta_smem > max_smem) return SQUANT_ERR_TOO_WIDE;
         if (cta_smem > p.smem_bytes) p.smem_bytes = static_cast<int>(cta_smem);
@@ -170,7 +168,7 @@ int build_param_plan(const squant_layer *layers, int32_t n_layers, const squant_
     std::vector<LayerDesc> descs(n_layers);
     std::vector<int> order(n_layers);
     for (int i = 0; i < n_layers; ++i) {
-        const int64_t cta_smem = layout_layer(layers[i], descs[i]);
+        const int64_t cta_smem = layout_layer(layers[i], descs[i], o.mode);
         if (cta_smem > max_smem) return SQUANT_ERR_TOO_WIDE;
         if (cta_smem > p.smem_bytes) p.smem_bytes = static_cast<int>(cta_smem);
         order[i] = i;
@@ -493,7 +491,7 @@ const char *squant_strerror(int code)
         case SQUANT_ERR_NULL: return "a required pointer is NULL";
         case SQUANT_ERR_SHAPE: return "a layer dimension is not positive or the element count overflows";
         case SQUANT_ERR_BITS: return "bits must be in 2..8 (2..4 with SQUANT_FLAG_PACK_INT4)";
-        case SQUANT_ERR_MODE: return "mode mask must contain E and be one of E, E|K, E|K|C (E|C only for 1x1 kernels); unknown flag bits are rejected";
+        case SQUANT_ERR_MODE: return "mode mask must contain E (E, E|K, E|C or E|K|C); unknown mode or flag bits are rejected";
         case SQUANT_ERR_ALIGN: return "float pointers must be 4-byte aligned";
         case SQUANT_ERR_TOO_WIDE: return "an output channel (cin*kh*kw) does not fit the on-chip path";
         case SQUANT_ERR_CUDA: return "a CUDA runtime call failed (see squant_last_cuda_error)";

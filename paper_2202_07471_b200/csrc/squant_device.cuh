@@ -733,6 +733,63 @@ __device__ __forceinline__ void channel_body(const LayerDesc &L, int m, const Gr
     emit_channel(L, m, G, reinterpret_cast<const unsigned char *>(cbuf), slice, s, ec, mode);
 }
 
+// ---------------------------------------------------------------- channel body, E + C without K
+// The E&C ablation of the paper's granularity study (Table 5): SQuant-K is left out, so every
+// ELEMENT of the channel is its own candidate for SQuant-C (Algorithm 2 on the channel with the
+// elements' perturbations as keys, ties by lower flat index).  The channel is handled as N*K
+// one-element kernels (the layer's slice is laid out that way); the kernels' error sums are
+// formed afterwards from the final perturbations.
+__device__ __forceinline__ void channel_body_ec(const LayerDesc &L, int m, const Group &G,
+                                                unsigned char *slice, float s, unsigned mode)
+{
+    const int N = L.N, K = L.K, NK = L.NK;
+    float *wbuf = reinterpret_cast<float *>(slice);
+    int *P = reinterpret_cast<int *>(slice);   // perturbations overwrite the weights
+    int8_t *cbuf = reinterpret_cast<int8_t *>(slice + L.off_codes);
+    int *hist = reinterpret_cast<int *>(slice + L.off_hist);
+    unsigned char *red = slice + L.off_red;
+    int *bc = reinterpret_cast<int *>(red + 128);
+    long long esum = 0;
+    for (int j = G.t; j < NK; j += G.g) {
+        int q, p;
+        squant_e(wbuf[j], s, q, p);
+        cbuf[j] = static_cast<int8_t>(q);
+        P[j] = p;
+        esum += p;
+    }
+    long long ec = group_sum(G, esum, red);   // barrier: perturbations and codes visible
+    if (ec != 0) {
+        const int sgn_c = ec > 0 ? 1 : -1;
+        const long long abs_e = ec > 0 ? ec : -ec;
+        const int kc = flip_count(abs_e);
+        if (kc > 0) {
+            unsigned long long T = ~0ull;
+            const int k_eff = select_threshold(G, P, NK, sgn_c, kc, hist, bc, T);
+            ec -= static_cast<long long>(sgn_c) * k_eff * kOne;
+            if (k_eff > 0) {
+                for (int j = G.t; j < NK; j += G.g) {
+                    const unsigned long long ck = cand_key(P[j], sgn_c, j);
+                    if (ck != 0 && ck >= T) {
+                        P[j] -= sgn_c * kOne;
+                        cbuf[j] = static_cast<int8_t>(cbuf[j] - sgn_c);
+                    }
+                }
+            }
+        }
+    }
+    G.sync();
+    if (L.kerr) {
+        float *kerr = L.kerr + static_cast<size_t>(m) * N;
+        for (int n = G.t; n < N; n += G.g) {
+            long long e = 0;
+            for (int i = 0; i < K; ++i) e += P[n * K + i];
+            kerr[n] = __fmul_rn(__ll2float_rn(e), 0x1p-30f);
+        }
+        G.sync();   // the perturbations are scratch for the packed emit
+    }
+    emit_channel(L, m, G, reinterpret_cast<const unsigned char *>(cbuf), slice, s, ec, mode);
+}
+
 // ---------------------------------------------------------------- channel body, 3x3 fast path
 // Needs K = 9, N a multiple of 4, SQuant-K in the mode mask and 2^-60 <= s <= 2^60.
 // A thread owns four consecutive kernels = 36 consecutive weights: nine conflict-free 128-bit
@@ -1082,7 +1139,9 @@ __device__ __forceinline__ void run_item(const LayerDesc &L, int ch0, unsigned c
     unsigned char *slice = smem + static_cast<size_t>(gi) * L.slice_bytes;
     const float s = stage_channel(L, m, G, slice, qmax);
     if (s == 0.0f) return;   // staging wait ran out (status word set); nothing is written
-    if (L.K == 1) {
+    if (L.K > 1 && (mode & 6u) == 4u) {   // E + C without K
+        channel_body_ec(L, m, G, slice, s, mode);
+    } else if (L.K == 1) {
         if ((L.N & 3) == 0 && s >= 0x1p-60f && s <= 0x1p60f)
             channel_body_k1_fast(L, m, G, slice, s, mode);
         else

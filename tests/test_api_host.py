@@ -50,7 +50,7 @@ def test_plan_geometry_for_the_five_configs():
     ((0, 3, 3, 3), {}, -2), ((4, -1, 3, 3), {}, -2), ((4, 3, 0, 3), {}, -2),
     ((4, 3, 3, 3), {"bits": 1}, -3), ((4, 3, 3, 3), {"bits": 9}, -3),
     ((4, 3, 3, 3), {"mode": 2}, -4), ((4, 3, 3, 3), {"mode": 8 | 1}, -4),
-    ((4, 3, 3, 3), {"mode": 1 | 4}, -4), ((4, 3, 3, 3), {"flags": 16}, -4),
+    ((4, 3, 3, 3), {"mode": 16 | 1}, -4), ((4, 3, 3, 3), {"flags": 16}, -4),
     ((4, 3, 3, 3), {"bits": 6, "flags": 3}, -3),
     ((4, 70000, 1, 1), {}, -6), ((4, 8000, 3, 3), {}, -6),
 ])
@@ -62,7 +62,8 @@ def test_invalid_arguments_are_rejected(shape, kw, code):
 
 def test_valid_edge_arguments():
     assert _info([], bits=4)["grid_ctas"] == 0
-    assert _info([(4, 300, 1, 1)], mode=1 | 4)["grid_ctas"] >= 1      # E|C is fine on 1x1 kernels
+    assert _info([(4, 300, 1, 1)], mode=1 | 4)["grid_ctas"] >= 1      # E|C ablation mode
+    assert _info([(4, 30, 3, 3)], mode=1 | 4)["grid_ctas"] >= 1
     assert _info([(1, 1, 1, 1)], bits=2)["grid_ctas"] == 1
     assert _info([(2, 4000, 3, 3)])["grid_ctas"] == 2
 

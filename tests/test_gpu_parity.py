@@ -48,14 +48,16 @@ def test_shape_sweep_grouped(bits):
     """Every sweep shape in ONE grouped launch: ragged tails, every kernel size path, all group
     sizes, special channels (zero, constant, tiny, huge, ties)."""
     ws = [adversarial_layer(s, seed=17 * bits + i) for i, s in enumerate(SWEEP_SHAPES)]
-    for mode in (EKC, EK, E):
+    for mode in (EKC, EK, E, sq.MODE_E | sq.MODE_C):
         bufs = run_gpu(ws, bits, mode)
         for i, (b, w) in enumerate(zip(bufs, ws)):
             assert_layer_equal(b, w, bits, mode, tag=f"shape{SWEEP_SHAPES[i]} mode{mode}")
 
 
-def test_e_c_mode_on_1x1():
-    ws = [adversarial_layer(s, seed=5) for s in [(7, 300, 1, 1), (4, 2049, 1, 1)]]
+def test_e_c_mode_without_k():
+    """The E&C ablation (Table 5 of the paper): every element is its own SQuant-C candidate."""
+    ws = [adversarial_layer(s, seed=5) for s in [(7, 300, 1, 1), (4, 2049, 1, 1), (6, 64, 3, 3), (3, 2048, 3, 3),
+                                                 (5, 7, 5, 5), (9, 1, 3, 3), (4, 3, 7, 7), (3, 33, 2, 2)]]
     mode = sq.MODE_E | sq.MODE_C
     bufs = run_gpu(ws, 4, mode)
     for b, w in zip(bufs, ws):
