@@ -124,15 +124,13 @@ __device__ __forceinline__ void bulk_store_wait()
 // `red` points at 16 eight-byte slots owned by the group.
 __device__ __forceinline__ float group_absmax(const Group &G, float v, void *red)
 {
+    // `slot` (red + 216) was zeroed before the previous group barrier
     unsigned u = __reduce_max_sync(kFull, __float_as_uint(v));  // v >= 0: uint order = float order
     if (G.g > 32) {
-        unsigned *r = reinterpret_cast<unsigned *>(red);
-        if ((G.t & 31) == 0) r[G.t >> 5] = u;
+        unsigned *slot = reinterpret_cast<unsigned *>(static_cast<unsigned char *>(red) + 216);
+        if ((G.t & 31) == 0) atomicMax(slot, u);
         G.sync();
-        const int nw = G.g >> 5;
-        u = 0;
-        for (int i = 0; i < nw; ++i) u = max(u, r[i]);
-        G.sync();
+        u = *slot;
     } else {
         __syncwarp();
     }
@@ -506,9 +504,12 @@ __device__ __forceinline__ bool kernel9_fast(const float (&Pf)[9], const float *
         m3 = max(m3, u);
         m4 = max(m4, x);
     }
+    // leading ranks whose truncated keys are strictly ordered (0..3); the decision needs
+    // (j + 2) / 2 of them: j = 0, 1 -> 1; 2, 3 -> 2; 4, 5 -> 3
     const bool d12 = (m1 >> 4) > (m2 >> 4), d23 = (m2 >> 4) > (m3 >> 4), d34 = (m3 >> 4) > (m4 >> 4);
+    const int certified = d12 ? (d23 ? (d34 ? 3 : 2) : 1) : 0;
     const bool zero = near & (j == 0) & (eabs == 0u);   // e == 0: no flips, no candidate
-    const bool ok = zero | (!near & d12 & ((j <= 1) | (d23 & ((j <= 3) | (d34 & (j <= 5))))));
+    const bool ok = zero | (!near & (j <= 5) & (certified >= ((j + 2) >> 1)));
     // ok with j >= 1 implies m1 >= 16, with j >= 2 m2 >= 16, with j >= 4 m3 >= 16: indices are 0..8
     if (ok & (j >= 1)) {
         const int i1 = ~m1 & 15;   // = 15 - (m1 & 15)
@@ -560,6 +561,7 @@ __device__ __forceinline__ float stage_channel(const LayerDesc &L, int m, const 
         if (G.t == 0) {
             reinterpret_cast<int *>(red + 128)[5] = 0;                    // boundary-list count
             *reinterpret_cast<unsigned long long *>(red + 208) = 0ull;   // channel-sum accumulator
+            *reinterpret_cast<unsigned *>(red + 216) = 0u;               // absmax slot
         }
     }
     if ((reinterpret_cast<uintptr_t>(wg) & 15) == 0 && (NK & 3) == 0) {
@@ -587,6 +589,7 @@ __device__ __forceinline__ float stage_channel(const LayerDesc &L, int m, const 
             wbuf[i] = t;
             amax = fmaxf(amax, fabsf(t));
         }
+        G.sync();   // the zeroed scratch is visible before the reduction uses it
         amax = group_absmax(G, amax, red);
     }
     return (amax < 0x1p-100f) ? 1.0f : __fdiv_rn(amax, static_cast<float>(qmax));
@@ -804,7 +807,7 @@ __device__ __forceinline__ void channel_body_ec(const LayerDesc &L, int m, const
 // kernels above it are flipped, the few inside it are collected in a list and ranked exactly
 // (|v| descending, kernel index ascending).  A boundary bin too crowded for the list (massive
 // ties) falls back to the general radix select.
-constexpr int kListCap = 256;
+constexpr int kListCap = 128;   // the boundary list lives in the histogram's 1 KB once the scan is done
 
 __device__ __forceinline__ void hist_add(int *hist, int v)
 {

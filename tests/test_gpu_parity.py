@@ -218,3 +218,18 @@ def test_packed_int4_output(bits):
         assert np.array_equal(b.kernel_err.cpu().numpy(), r.kernel_err)
     with pytest.raises(sq.SquantError):
         sq.squant_quantize_model(bufs[:1], bits=8, flags=flags)
+
+
+@pytest.mark.parametrize("k", [1, 9])
+def test_boundary_bin_between_list_and_radix_capacity(k):
+    """SQuant-C boundary bins of every size class: taken whole, ranked from the short list
+    (<= 128 members), and the radix-select fallback (129..256 and thousands of tied members)."""
+    for members in (40, 128, 129, 200, 256, 257, 700):
+        n = 1024
+        w = np.zeros((2, n, k), dtype=np.float32)
+        w[:, 0, 0] = 127.0                         # scale 1 with bits = 8
+        w[:, 1:51, 0] = 0.45                       # 50 candidates at -0.45: taken whole
+        w[:, 51:51 + members, 0] = 0.30            # `members` tied candidates at -0.30: boundary bin
+        w[1] = -w[1]
+        (b,) = run_gpu([w.reshape(2, n, 3, 3) if k == 9 else w.reshape(2, n, 1, 1)], 8, EKC)
+        assert_layer_equal(b, w.reshape(2, n, 3, 3) if k == 9 else w.reshape(2, n, 1, 1), 8, EKC, tag=f"members {members}")
