@@ -681,7 +681,7 @@ __device__ __forceinline__ void channel_body(const LayerDesc &L, int m, const Gr
 
     // ---- SQuant-E, SQuant-K, candidate: one thread per kernel
     // Without SQuant-K a kernel sum can reach K/2 and no longer fits 32 bits; it is then
-    // emitted right here (no channel step follows: E|C is only accepted for 1x1 kernels).
+    // emitted right here (no channel step follows: E|C on larger kernels has its own body).
     const bool do_k = (mode & 2u) != 0;
     const bool keep = do_k || KT == 1 || K == 1;
     float *kerr = L.kerr ? L.kerr + static_cast<size_t>(m) * N : nullptr;
@@ -793,26 +793,13 @@ __device__ __forceinline__ void channel_body_ec(const LayerDesc &L, int m, const
     emit_channel(L, m, G, reinterpret_cast<const unsigned char *>(cbuf), slice, s, ec, mode);
 }
 
-// ---------------------------------------------------------------- channel body, 3x3 fast path
-// Needs K = 9, N a multiple of 4, SQuant-K in the mode mask and 2^-60 <= s <= 2^60.
-// A thread owns four consecutive kernels = 36 consecutive weights: nine conflict-free 128-bit
-// shared loads in, nine conflict-free 32-bit stores of packed code bytes out; flips are byte
-// read-modify-writes on the staged codes.  Kernel error sums are written as soon as SQuant-K is
-// done; SQuant-C later patches the few kernels it flips.
-//
-// SQuant-C needs ONE histogram, filled while the kernels are processed: bin = |v| >> 22 of each
-// kernel's candidate, positive and negative candidates counted in the two halves of one 32-bit
-// word.  Once the channel sum (hence the sign and k_c) is known, one warp scans the histogram
-// of that sign for the boundary bin;
-// kernels above it are flipped, the few inside it are collected in a list and ranked exactly
-// (|v| descending, kernel index ascending).  A boundary bin too crowded for the list (massive
-// ties) falls back to the general radix select.
+// ---------------------------------------------------------------- SQuant-C by histogram (fast paths)
 constexpr int kListCap = 128;   // the boundary list lives in the histogram's 1 KB once the scan is done
 
 __device__ __forceinline__ void hist_add(int *hist, int v)
 {
-    const int a = v < 0 ? -v : v;                           // < 2^30: bin < 256
-    atomicAdd(&hist[a >> 22], (v > 0 ? 1 : 0) | (v < 0 ? 0x10000 : 0));
+    const int a = v < 0 ? -v : v;   // < 2^30 for every valid candidate; clamped for garbage input
+    atomicAdd(&hist[min(a >> 22, kHistBins - 1)], (v > 0 ? 1 : 0) | (v < 0 ? 0x10000 : 0));
 }
 
 // Second half of a fast-path channel: channel sum, SQuant-C by the candidate histogram, flips,
@@ -958,8 +945,20 @@ __device__ __forceinline__ void finish_channel_hist(const LayerDesc &L, int m, c
     emit_channel(L, m, G, cbuf, slice, s, ec, mode);
 }
 
-
-
+// ---------------------------------------------------------------- channel body, 3x3 fast path
+// Needs K = 9, N a multiple of 4, SQuant-K in the mode mask and 2^-60 <= s <= 2^60.
+// A thread owns four consecutive kernels = 36 consecutive weights: nine conflict-free 128-bit
+// shared loads in, nine conflict-free 32-bit stores of packed code bytes out; flips are byte
+// read-modify-writes on the staged codes.  Kernel error sums are written as soon as SQuant-K is
+// done; SQuant-C later patches the few kernels it flips.
+//
+// SQuant-C needs ONE histogram, filled while the kernels are processed: bin = |v| >> 22 of each
+// kernel's candidate, positive and negative candidates counted in the two halves of one 32-bit
+// word.  Once the channel sum (hence the sign and k_c) is known, one warp scans the histogram
+// of that sign for the boundary bin;
+// kernels above it are flipped, the few inside it are collected in a list and ranked exactly
+// (|v| descending, kernel index ascending).  A boundary bin too crowded for the list (massive
+// ties) falls back to the general radix select.
 __device__ __forceinline__ void channel_body_k9_fast(const LayerDesc &L, int m, const Group &G,
                                                      unsigned char *slice, float s, unsigned mode)
 {
