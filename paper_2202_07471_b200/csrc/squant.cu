@@ -173,10 +173,14 @@ int build_param_plan(const squant_layer *layers, int32_t n_layers, const squant_
         if (cta_smem > p.smem_bytes) p.smem_bytes = static_cast<int>(cta_smem);
         order[i] = i;
     }
+    // Estimated duration of one CTA of the layer.  Kernel sizes other than 1x1 and 3x3 take the
+    // general per-thread path, which is latency-bound and far slower per weight (a 7x7 stem CTA
+    // is the longest of a whole ResNet), so those start first.
     auto cta_work = [&](int i) {
         const LayerDesc &d = descs[i];
         const int64_t groups = sq::kCtaThreads / d.g;
-        return (groups < d.M ? groups : d.M) * static_cast<int64_t>(d.NK);
+        const int64_t per_channel = (d.K == 1 || d.K == 9) ? d.NK : static_cast<int64_t>(d.NK) * 64 * d.K;
+        return (groups < d.M ? groups : d.M) * per_channel;
     };
     std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return cta_work(a) > cta_work(b); });
     for (int base = 0; base < n_layers; base += sq::kMaxParamLayers) {
