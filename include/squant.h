@@ -93,6 +93,8 @@ typedef struct squant_layer {
                                  perturbations, (float)(integer sum) * 2^-30 */
     float *channel_err;  /* out, may be NULL: [cout] final signed sum of a channel's
                                  perturbations */
+    float *dequant;      /* out, may be NULL: [cout][cin][kh][kw] fp32 quantized weights
+                                 code * s_m - what Algorithm 1 itself returns ("C * s") */
 } squant_layer;
 
 /*

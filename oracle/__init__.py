@@ -37,7 +37,7 @@ def _load():
         lib.sqo_quantize_layer.argtypes = [
             ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
             ctypes.POINTER(_Options), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
-            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
         _lib = lib
     return _lib
 
@@ -50,6 +50,7 @@ class OracleResult:
     channel_err: np.ndarray                # fp32 [M]
     pert: Optional[np.ndarray] = None      # int32 fixed-point perturbations (2^-30 units)
     flip: Optional[np.ndarray] = None      # uint8: bit0 flipped by SQuant-K, bit1 by SQuant-C
+    dequant: Optional[np.ndarray] = None   # fp32 code * scale (what Algorithm 1 returns)
 
 
 def quantize_layer(w: np.ndarray, bits: int = 4, mode: int = MODE_EKC,
@@ -69,10 +70,11 @@ def quantize_layer(w: np.ndarray, bits: int = 4, mode: int = MODE_EKC,
     cerr = np.empty(M, dtype=np.float32)
     pert = np.empty(w.shape, dtype=np.int32) if details else None
     flip = np.empty(w.shape, dtype=np.uint8) if details else None
+    deq = np.empty(w.shape, dtype=np.float32) if details else None
     opt = _Options(bits, mode, flags)
     ptr = lambda a: a.ctypes.data_as(ctypes.c_void_p) if a is not None else None
     rc = _load().sqo_quantize_layer(ptr(w), M, N, K, ctypes.byref(opt), ptr(codes), ptr(scales),
-                                    ptr(kerr), ptr(cerr), ptr(pert), ptr(flip))
+                                    ptr(kerr), ptr(cerr), ptr(pert), ptr(flip), ptr(deq))
     if rc != 0:
         raise ValueError(f"sqo_quantize_layer failed with code {rc}")
-    return OracleResult(codes, scales, kerr, cerr, pert, flip)
+    return OracleResult(codes, scales, kerr, cerr, pert, flip, deq)

@@ -104,7 +104,7 @@ typedef struct {
 
 static void sqo_channel(const float *w, int32_t N, int32_t K, const sqo_options *opt,
                         sqo_work *wk, int8_t *codes, float *scale_out,
-                        float *kernel_err, float *channel_err)
+                        float *kernel_err, float *channel_err, float *dequant)
 {
     const int32_t NK = N * K;
     const int32_t qmax = (1 << (opt->bits - 1)) - 1;
@@ -219,6 +219,8 @@ static void sqo_channel(const float *w, int32_t N, int32_t K, const sqo_options 
         if (kernel_err) kernel_err[n] = (float)e * 0x1p-30f;
     }
     if (channel_err) *channel_err = (float)total * 0x1p-30f;
+    if (dequant)   /* what Algorithm 1 returns: C * s */
+        for (int32_t j = 0; j < NK; ++j) dequant[j] = (float)q[j] * s;
     if (opt->flags & SQO_FLAG_PACK_INT4) {
         for (int32_t j = 0; j < NK; j += 2) {
             unsigned lo = (unsigned)q[j] & 15u;
@@ -239,11 +241,12 @@ static void sqo_channel(const float *w, int32_t N, int32_t K, const sqo_options 
  *   channel_err  out [M], may be NULL
  *   pert         out [M][N][K] final fixed-point perturbations (2^-30 units), may be NULL
  *   flip         out [M][N][K] flip record (bit0 SQuant-K, bit1 SQuant-C), may be NULL
+ *   dequant      out [M][N][K] fp32 code * scale (Algorithm 1's return value), may be NULL
  * Inputs must be finite.  Returns SQO_OK or a negative error.
  */
 int sqo_quantize_layer(const float *w, int32_t M, int32_t N, int32_t K, const sqo_options *opt,
                        int8_t *codes, float *scales, float *kernel_err, float *channel_err,
-                       int32_t *pert, uint8_t *flip)
+                       int32_t *pert, uint8_t *flip, float *dequant)
 {
     if (!w || !opt || !codes || !scales || M < 0 || N <= 0 || K <= 0) return SQO_ERR_ARG;
     if (opt->bits < 2 || opt->bits > 8 || !(opt->mode & SQO_MODE_E)) return SQO_ERR_ARG;
@@ -265,7 +268,8 @@ int sqo_quantize_layer(const float *w, int32_t M, int32_t N, int32_t K, const sq
             sqo_channel(w + (size_t)m * NK, N, K, opt, &wk,
                         codes + (size_t)m * ((opt->flags & SQO_FLAG_PACK_INT4) ? (NK + 1) / 2 : NK), scales + m,
                         kernel_err ? kernel_err + (size_t)m * N : NULL,
-                        channel_err ? channel_err + m : NULL);
+                        channel_err ? channel_err + m : NULL,
+                        dequant ? dequant + (size_t)m * NK : NULL);
             if (pert) memcpy(pert + (size_t)m * NK, wk.P, NK * sizeof(int32_t));
             if (flip) memcpy(flip + (size_t)m * NK, wk.flip, NK);
         }

@@ -41,7 +41,7 @@ class Layer(ctypes.Structure):
     _fields_ = [("w", ctypes.c_void_p), ("cout", ctypes.c_int32), ("cin", ctypes.c_int32),
                 ("kh", ctypes.c_int32), ("kw", ctypes.c_int32), ("codes", ctypes.c_void_p),
                 ("scales", ctypes.c_void_p), ("kernel_err", ctypes.c_void_p),
-                ("channel_err", ctypes.c_void_p)]
+                ("channel_err", ctypes.c_void_p), ("dequant", ctypes.c_void_p)]
 
 
 _lib = None
@@ -91,10 +91,11 @@ class LayerBuffers:
     scales: torch.Tensor
     kernel_err: Optional[torch.Tensor]
     channel_err: Optional[torch.Tensor]
+    dequant: Optional[torch.Tensor] = None     # fp32 code * scale, shape of the weights
 
 
 def alloc_outputs(w: torch.Tensor, kernel_err: bool = True, channel_err: bool = True,
-                  pin: bool = False, pack_int4: bool = False) -> LayerBuffers:
+                  pin: bool = False, pack_int4: bool = False, dequant: bool = False) -> LayerBuffers:
     """Allocate output tensors next to `w` ([cout, cin, kh, kw], [cout, cin, k] or [cout, cin]).
     With pack_int4 the codes tensor is [cout, ceil(cin*kh*kw / 2)] (for FLAG_PACK_INT4)."""
     if w.dtype != torch.float32 or not w.is_contiguous() or w.dim() < 2:
@@ -107,7 +108,8 @@ def alloc_outputs(w: torch.Tensor, kernel_err: bool = True, channel_err: bool = 
     return LayerBuffers(
         w, torch.empty(cshape, dtype=torch.int8, **kw), torch.empty(m, dtype=torch.float32, **kw),
         torch.empty((m, n), dtype=torch.float32, **kw) if kernel_err else None,
-        torch.empty(m, dtype=torch.float32, **kw) if channel_err else None)
+        torch.empty(m, dtype=torch.float32, **kw) if channel_err else None,
+        torch.empty(w.shape, dtype=torch.float32, **kw) if dequant else None)
 
 
 def _descriptor(b: LayerBuffers) -> Layer:
@@ -122,7 +124,7 @@ def _descriptor(b: LayerBuffers) -> Layer:
     else:
         raise ValueError("weights must be [cout, cin], [cout, cin, k] or [cout, cin, kh, kw]")
     ptr = lambda t: t.data_ptr() if t is not None else None
-    return Layer(ptr(w), m, n, kh, kw, ptr(b.codes), ptr(b.scales), ptr(b.kernel_err), ptr(b.channel_err))
+    return Layer(ptr(w), m, n, kh, kw, ptr(b.codes), ptr(b.scales), ptr(b.kernel_err), ptr(b.channel_err), ptr(b.dequant))
 
 
 def _options(bits: int, mode: int, flags: int) -> Options:
@@ -207,7 +209,7 @@ def squant_plan_info(shapes: Sequence[Sequence[int]], bits: int = 4, mode: int =
                      flags: int = FLAG_NARROW_RANGE) -> dict:
     """Launch geometry for layers of the given [cout, cin, kh, kw] shapes (no GPU needed)."""
     arr = (Layer * max(1, len(shapes)))(*[Layer(None, int(s[0]), int(s[1]), int(s[2]), int(s[3]),
-                                                None, None, None, None) for s in shapes])
+                                                None, None, None, None, None) for s in shapes])
     opt = _options(bits, mode, flags)
     g, t, s = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32()
     _check(load_library().squant_plan_info(arr, len(shapes), ctypes.byref(opt), ctypes.byref(g),

@@ -88,7 +88,7 @@ int validate(const squant_layer *layers, int32_t n_layers, const squant_options 
             if (!l.w || !l.codes || !l.scales) return SQUANT_ERR_NULL;
             if ((reinterpret_cast<uintptr_t>(l.w) & 3) || (reinterpret_cast<uintptr_t>(l.scales) & 3) ||
                 (reinterpret_cast<uintptr_t>(l.kernel_err) & 3) ||
-                (reinterpret_cast<uintptr_t>(l.channel_err) & 3))
+                (reinterpret_cast<uintptr_t>(l.channel_err) & 3) || (reinterpret_cast<uintptr_t>(l.dequant) & 3))
                 return SQUANT_ERR_ALIGN;
         }
     }
@@ -99,7 +99,7 @@ int validate(const squant_layer *layers, int32_t n_layers, const squant_options 
 // slice.  Returns the dynamic shared memory one CTA needs for this layer.
 int64_t layout_layer(const squant_layer &l, LayerDesc &d, unsigned mode)
 {
-    d.w = l.w; d.codes = l.codes; d.scales = l.scales; d.kerr = l.kernel_err; d.cerr = l.channel_err;
+    d.w = l.w; d.codes = l.codes; d.scales = l.scales; d.kerr = l.kernel_err; d.cerr = l.channel_err; d.deq = l.dequant;
     d.M = l.cout; d.N = l.cin; d.K = l.kh * l.kw; d.NK = d.N * d.K;
     d.g = group_size(d.NK);
     d.g_shift = 0;
@@ -340,18 +340,19 @@ int squant_quantize_model_host(const squant_layer *layers, int32_t n_layers,
     SQ_CUDA(cudaGetDevice(&device));
     // carve one device arena: per layer weights, codes, scales, kernel sums, channel sums
     std::vector<squant_layer> dev(layers, layers + n_layers);
-    std::vector<size_t> off(static_cast<size_t>(n_layers) * 5);
+    std::vector<size_t> off(static_cast<size_t>(n_layers) * 6);
     size_t total = 0;
     for (int i = 0; i < n_layers; ++i) {
         const squant_layer &l = layers[i];
         const size_t n = static_cast<size_t>(l.cin) * l.kh * l.kw * l.cout;
-        off[5 * i + 0] = total; total += align256(n * 4);
+        off[6 * i + 0] = total; total += align256(n * 4);
         const size_t code_bytes = (o.flags & SQUANT_FLAG_PACK_INT4)
                                       ? static_cast<size_t>(l.cout) * ((static_cast<size_t>(l.cin) * l.kh * l.kw + 1) / 2) : n;
-        off[5 * i + 1] = total; total += align256(code_bytes);
-        off[5 * i + 2] = total; total += align256(static_cast<size_t>(l.cout) * 4);
-        off[5 * i + 3] = total; total += l.kernel_err ? align256(static_cast<size_t>(l.cout) * l.cin * 4) : 0;
-        off[5 * i + 4] = total; total += l.channel_err ? align256(static_cast<size_t>(l.cout) * 4) : 0;
+        off[6 * i + 1] = total; total += align256(code_bytes);
+        off[6 * i + 2] = total; total += align256(static_cast<size_t>(l.cout) * 4);
+        off[6 * i + 3] = total; total += l.kernel_err ? align256(static_cast<size_t>(l.cout) * l.cin * 4) : 0;
+        off[6 * i + 4] = total; total += l.channel_err ? align256(static_cast<size_t>(l.cout) * 4) : 0;
+        off[6 * i + 5] = total; total += l.dequant ? align256(n * 4) : 0;
     }
     if (static_cast<int>(g_arenas.size()) <= device) g_arenas.resize(device + 1);
     Arena &a = g_arenas[device];
@@ -365,12 +366,13 @@ int squant_quantize_model_host(const squant_layer *layers, int32_t n_layers,
     for (int i = 0; i < n_layers; ++i) {
         const squant_layer &l = layers[i];
         const size_t n = static_cast<size_t>(l.cin) * l.kh * l.kw * l.cout;
-        dev[i].w = reinterpret_cast<const float *>(base + off[5 * i + 0]);
-        dev[i].codes = reinterpret_cast<int8_t *>(base + off[5 * i + 1]);
-        dev[i].scales = reinterpret_cast<float *>(base + off[5 * i + 2]);
-        dev[i].kernel_err = l.kernel_err ? reinterpret_cast<float *>(base + off[5 * i + 3]) : nullptr;
-        dev[i].channel_err = l.channel_err ? reinterpret_cast<float *>(base + off[5 * i + 4]) : nullptr;
-        SQ_CUDA(cudaMemcpyAsync(base + off[5 * i + 0], l.w, n * 4, cudaMemcpyHostToDevice, stream));
+        dev[i].w = reinterpret_cast<const float *>(base + off[6 * i + 0]);
+        dev[i].codes = reinterpret_cast<int8_t *>(base + off[6 * i + 1]);
+        dev[i].scales = reinterpret_cast<float *>(base + off[6 * i + 2]);
+        dev[i].kernel_err = l.kernel_err ? reinterpret_cast<float *>(base + off[6 * i + 3]) : nullptr;
+        dev[i].channel_err = l.channel_err ? reinterpret_cast<float *>(base + off[6 * i + 4]) : nullptr;
+        dev[i].dequant = l.dequant ? reinterpret_cast<float *>(base + off[6 * i + 5]) : nullptr;
+        SQ_CUDA(cudaMemcpyAsync(base + off[6 * i + 0], l.w, n * 4, cudaMemcpyHostToDevice, stream));
     }
     const ParamPlan *pp = nullptr;
     rc = get_plan(dev.data(), n_layers, o, pp);
@@ -388,6 +390,8 @@ int squant_quantize_model_host(const squant_layer *layers, int32_t n_layers,
             SQ_CUDA(cudaMemcpyAsync(l.kernel_err, dev[i].kernel_err, static_cast<size_t>(l.cout) * l.cin * 4, cudaMemcpyDeviceToHost, stream));
         if (l.channel_err)
             SQ_CUDA(cudaMemcpyAsync(l.channel_err, dev[i].channel_err, static_cast<size_t>(l.cout) * 4, cudaMemcpyDeviceToHost, stream));
+        if (l.dequant)
+            SQ_CUDA(cudaMemcpyAsync(l.dequant, dev[i].dequant, n * 4, cudaMemcpyDeviceToHost, stream));
     }
     SQ_CUDA(cudaStreamSynchronize(stream));
     return SQUANT_OK;

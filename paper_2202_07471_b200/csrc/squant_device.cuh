@@ -29,6 +29,7 @@ struct LayerDesc {
     float *scales;
     float *kerr;
     float *cerr;
+    float *deq;
     int32_t M, N, K, NK;
     int32_t g;            // threads per channel group: 32, 64, 128, 256 or 512
     int32_t g_shift;      // log2(g)
@@ -637,6 +638,23 @@ __device__ __forceinline__ void emit_channel(const LayerDesc &L, int m, const Gr
                                              long long ec, unsigned mode)
 {
     const int NK = L.NK;
+    if (L.deq) {   // Algorithm 1's own return value: code * s, fp32
+        float *dg = L.deq + static_cast<size_t>(m) * NK;
+        if ((reinterpret_cast<uintptr_t>(dg) & 15) == 0 && (NK & 3) == 0) {
+            for (int i = G.t; i < (NK >> 2); i += G.g) {
+                const unsigned c4 = reinterpret_cast<const unsigned *>(cbuf)[i];
+                float4 f;
+                f.x = __fmul_rn(__int2float_rn(static_cast<signed char>(c4 & 255u)), s);
+                f.y = __fmul_rn(__int2float_rn(static_cast<signed char>((c4 >> 8) & 255u)), s);
+                f.z = __fmul_rn(__int2float_rn(static_cast<signed char>((c4 >> 16) & 255u)), s);
+                f.w = __fmul_rn(__int2float_rn(static_cast<signed char>(c4 >> 24)), s);
+                __stcs(reinterpret_cast<float4 *>(dg) + i, f);
+            }
+        } else {
+            for (int i = G.t; i < NK; i += G.g)
+                dg[i] = __fmul_rn(__int2float_rn(static_cast<signed char>(cbuf[i])), s);
+        }
+    }
     const unsigned char *src = cbuf;
     int row = NK;
     if (mode & kModePackInt4) {

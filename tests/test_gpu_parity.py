@@ -233,3 +233,19 @@ def test_boundary_bin_between_list_and_radix_capacity(k):
         w[1] = -w[1]
         (b,) = run_gpu([w.reshape(2, n, 3, 3) if k == 9 else w.reshape(2, n, 1, 1)], 8, EKC)
         assert_layer_equal(b, w.reshape(2, n, 3, 3) if k == 9 else w.reshape(2, n, 1, 1), 8, EKC, tag=f"members {members}")
+
+
+def test_dequantized_output():
+    """Optional fp32 output code * s (what Algorithm 1 returns), all paths, aligned and not."""
+    shapes = [(6, 64, 3, 3), (3, 2048, 3, 3), (5, 256, 1, 1), (7, 33, 1, 1), (4, 3, 5, 5), (3, 7, 3, 3)]
+    ws = [adversarial_layer(s, seed=40 + i) for i, s in enumerate(shapes)]
+    for flags, pack in ((sq.FLAG_NARROW_RANGE, False), (sq.FLAG_NARROW_RANGE | sq.FLAG_PACK_INT4, True)):
+        bufs = [sq.alloc_outputs(torch.from_numpy(w).cuda(), dequant=True, pack_int4=pack) for w in ws]
+        for b in bufs:
+            b.dequant.fill_(float("nan"))
+        sq.squant_quantize_model(bufs, bits=4, mode=EKC, flags=flags)
+        sq.squant_device_status()
+        for b, w, shp in zip(bufs, ws, shapes):
+            r = oracle.quantize_layer(w, bits=4, mode=EKC, flags=flags, details=True)
+            assert np.array_equal(b.dequant.cpu().numpy().view(np.uint32), r.dequant.view(np.uint32)), f"shape {shp}"
+            assert np.array_equal(b.codes.cpu().numpy(), r.codes)

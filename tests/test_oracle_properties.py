@@ -407,3 +407,16 @@ def test_packed_int4_output_is_a_relabelling(shape, bits):
         assert not ((b.codes[:, -1].astype(np.uint8) >> 4).any())   # pad nibble is zero
     with pytest.raises(ValueError):
         oracle.quantize_layer(w, bits=6, flags=oracle.FLAG_PACK_INT4)
+
+
+@pytest.mark.parametrize("bits", [4, 8])
+def test_dequantized_output_is_code_times_scale(bits):
+    """Algorithm 1 returns C * s.  Every quantized weight is within one step of the original
+    (Eq. 12: |perturbation| < 1 in units of s), un-flipped ones within half a step."""
+    w = _layer((6, 20, 3, 3), seed=bits)
+    r = oracle.quantize_layer(w, bits=bits, mode=EKC, details=True)
+    s = r.scales[:, None, None, None]
+    assert np.array_equal(r.dequant, r.codes.astype(np.float32) * s)
+    err = np.abs(r.dequant.astype(np.float64) - w) / s
+    assert err.max() < 1.0 + 1e-6
+    assert err[r.flip == 0].max() <= 0.5 + 1e-6
