@@ -119,6 +119,23 @@ def mobilenetv2_shapes() -> List[Shape]:
     return s
 
 
+def mixed_kernel_shapes() -> List[Shape]:
+    """A synthetic family (not a published architecture) with the kernel shapes of
+    Inception / SqueezeNext / ShuffleNet style networks: factorised 1x7 / 7x1 / 1x3 / 3x1
+    convolutions, 5x5 and 3x3 convolutions, grouped convolutions (few input channels per kernel
+    group), pointwise layers and a classifier; 64 layers."""
+    s: List[Shape] = [(32, 3, 3, 3), (32, 32, 3, 3), (64, 32, 3, 3), (80, 64, 1, 1), (192, 80, 3, 3)]
+    for c in (192, 256, 288):
+        s += [(64, c, 1, 1), (48, c, 1, 1), (64, 48, 5, 5), (64, c, 1, 1), (96, 64, 3, 3), (96, 96, 3, 3)]
+    for c in (128, 160, 192):
+        s += [(192, 768, 1, 1), (c, 768, 1, 1), (c, c, 1, 7), (192, c, 7, 1), (c, c, 7, 1), (192, c, 1, 7)]
+    s += [(320, 1280, 1, 1), (384, 1280, 1, 1), (384, 384, 1, 3), (384, 384, 3, 1), (448, 1280, 1, 1), (384, 448, 3, 3)]
+    for c, g in ((240, 3), (480, 4), (960, 8)):          # grouped: cin per group = c / g
+        s += [(c, c // g, 1, 1), (c, 1, 3, 3), (c, c // g, 1, 1), (c // 2, c // (2 * g), 3, 1), (c // 2, c // (2 * g), 1, 3)]
+    s += [(1000, 2048, 1, 1), (1001, 1537, 1, 1)]
+    return s
+
+
 def large_layer_shapes() -> List[Shape]:
     return [(2048, 2048, 3, 3)] * 8
 
@@ -146,6 +163,7 @@ WORKLOADS = {
     "resnet18": Workload("resnet18", 2, tuple(resnet18_shapes()), "normal_laplace", (4,)),
     "resnet50": Workload("resnet50", 3, tuple(resnet50_shapes()), "student_t4", (4, 6)),
     "mobilenetv2": Workload("mobilenetv2", 4, tuple(mobilenetv2_shapes()), "normal", (4,)),
+    "mixed_kernels": Workload("mixed_kernels", 6, tuple(mixed_kernel_shapes()), "normal_laplace", (4,)),
     "large_layer": Workload("large_layer", 5, tuple(large_layer_shapes()), "normal_chanscale", (4,)),
 }
 

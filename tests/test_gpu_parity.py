@@ -99,7 +99,8 @@ def test_coarse_grid_ties_large_channel():
     assert_layer_equal(b, w, 8, EKC)
 
 
-@pytest.mark.parametrize("name,bits", [("resnet18", 4), ("resnet50", 4), ("resnet50", 6), ("mobilenetv2", 4)])
+@pytest.mark.parametrize("name,bits", [("resnet18", 4), ("resnet50", 4), ("resnet50", 6), ("mobilenetv2", 4),
+                                       ("mixed_kernels", 4)])
 def test_model_configs_full(name, bits):
     """Configs 2-4 at full size, the whole model in one grouped launch, every element compared."""
     wl = W.WORKLOADS[name]
