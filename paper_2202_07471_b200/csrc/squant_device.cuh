@@ -463,79 +463,77 @@ __device__ __noinline__ KernelOut kernel9_exact(const float *wk, float y, float 
 
 // Fast SQuant-K + Algorithm 3 on one 3x3 kernel whose exact perturbations Pf[0..8] (floats, in
 // 2^-30 units, before the conversion to integers) are in registers and whose code bytes are
-// already staged at cb.  Straight-line on purpose: every lane runs the same instructions and
-// the rare hand-back to kernel9_exact is a returned flag.
+// already staged at cb.  Straight-line on purpose: every lane runs the same instructions; a
+// kernel it cannot settle is reported (return value true) and redone by kernel9_exact.
 //
-// Sign, flip count and Over/Under come from a float sum of the perturbations.  That sum is
-// within 4096 units of the exact integer sum e (nine conversions round by <= 0.5 each, eight
-// additions by <= 256 each), and every decision boundary - 0, (j - 1/2) * 2^30 for k, j * 2^30 for
-// Over - is a multiple of 2^29; so with v = |sum| / 2^29 the decisions are exact whenever v is at
-// least 2^-17 away from an integer, and j = floor(v) gives k = (j + 1) / 2 and Over = (j odd).
-// Closer than that the kernel is handed back (an exactly zero integer sum is recognised first).
-// The exact |e| is still summed in integers (mod 2^32) for the error sum that is emitted.
+// Sign.  A float sum of the perturbations (within 4096 units of the exact sum) gives the sign
+// used to normalise the elements; the exact |e| is then the integer sum of the normalised
+// elements (mod 2^32).  If the float sign was wrong (|e| <= 4096) that sum wraps to >= 2^32 -
+// 4096 and the kernel is reported; |float sum| >= 3.75 * 2^30 (where 32 bits could wrap) too.
 //
-// Selection: keys are the sign-normalised integer perturbations with the element index folded
-// into their low four bits, (P & ~15) | (15 - i), so the four largest can be tracked by value
-// alone and carry their positions.  This orders by (P >> 4, index); it equals Algorithm 2's
-// order (P, index) whenever the truncated values of neighbouring ranks differ, which is checked.
-// Handled: j = 0..5, i.e. k = 0, 1, 2 and k = 3 when it is Over SQuant.
-__device__ __forceinline__ bool kernel9_fast(const float (&Pf)[9], const float *wk, float y, float s2,
-                                             unsigned char *cb, int &e_out, int &v_out, int &idx_out)
+// Decisions, all from the exact |e|: jx = (|e| - t) >> 29 with t = (|e| is no multiple of 2^30),
+// i.e. floor(|e| / 2^29) with "exactly k + 1/2" falling to the lower value.  Then the flip count
+// of Algorithm 2 is k = (jx + 1) / 2, the kernel is Over SQuant iff jx is odd, and the candidate
+// of Algorithm 3 is the element of rank c = (jx + 2) / 2 (the last flipped one when Over, the
+// first un-flipped one otherwise).  jx <= 5 is handled (k <= 3, c <= 3).
+//
+// Selection.  Keys are the sign-normalised integer perturbations with the element index folded
+// into their low four bits, (P & ~15) | (15 - i): distinct, and ordered like Algorithm 2's
+// (P descending, index ascending) among elements whose low four bits are zero.  That holds for
+// every element with P >= 2^27: its quotient w/s * 2^30 is an fp32 number of magnitude >= 2^27,
+// hence a multiple of 16.  So if the key of rank c is >= 2^27 the first c ranks are exact, and
+// so is the candidate's value (the key without its index bits); otherwise the kernel is
+// reported.  The three largest keys come from a 3x3 sorting tableau: sort each triple, then
+// the column of maxima; the top three of nine lie in row 1 and column 1 (21 operations).
+__device__ __forceinline__ bool kernel9_select(const float (&Pf)[9], unsigned char *cb, int &e_out,
+                                               int &v_out, unsigned &idx_out)
 {
     const float ef = __fadd_rn(__fadd_rn(__fadd_rn(__fadd_rn(Pf[0], Pf[1]), __fadd_rn(Pf[2], Pf[3])),
                                          __fadd_rn(__fadd_rn(Pf[4], Pf[5]), __fadd_rn(Pf[6], Pf[7]))),
                                Pf[8]);
     const float sgn_f = copysignf(1.0f, ef);
-    const int sgn = ef < 0.0f ? -1 : 1;
-    const float v = __fmul_rn(fabsf(ef), 0x1p-29f);
-    const bool near = fabsf(__fsub_rn(v, rintf(v))) < 0x1p-17f;
-    const int j = __float2int_rd(v);
-    int m1 = 0, m2 = 0, m3 = 0, m4 = 0;
+    const int sgn = (__float_as_int(ef) >> 31) | 1;
+    int a[9];
     unsigned eabs = 0;   // |e| mod 2^32
 #pragma unroll
     for (int i = 0; i < 9; ++i) {
         const int Ps = __float2int_rn(__fmul_rn(Pf[i], sgn_f));
         eabs += static_cast<unsigned>(Ps);
-        const int key = (Ps & ~15) | (15 - i);
-        const int t = min(m1, key);
-        m1 = max(m1, key);
-        const int u = min(m2, t);
-        m2 = max(m2, t);
-        const int x = min(m3, u);
-        m3 = max(m3, u);
-        m4 = max(m4, x);
+        a[i] = (Ps & ~15) | (15 - i);
     }
-    // leading ranks whose truncated keys are strictly ordered (0..3); the decision needs
-    // (j + 2) / 2 of them: j = 0, 1 -> 1; 2, 3 -> 2; 4, 5 -> 3
-    const bool d12 = (m1 >> 4) > (m2 >> 4), d23 = (m2 >> 4) > (m3 >> 4), d34 = (m3 >> 4) > (m4 >> 4);
-    const int certified = d12 ? (d23 ? (d34 ? 3 : 2) : 1) : 0;
-    const bool zero = near & (j == 0) & (eabs == 0u);   // e == 0: no flips, no candidate
-    const bool ok = zero | (!near & (j <= 5) & (certified >= ((j + 2) >> 1)));
-    // ok with j >= 1 implies m1 >= 16, with j >= 2 m2 >= 16, with j >= 4 m3 >= 16: indices are 0..8
-    if (ok & (j >= 1)) {
+    // |key| < 2^29 + 2^14, so the sum of three keys fits 32 bits: middle = sum - max - min
+    const int h1 = __vimax3_s32(a[0], a[1], a[2]), l1 = __vimin3_s32(a[0], a[1], a[2]), d1 = a[0] + a[1] + a[2] - h1 - l1;
+    const int h2 = __vimax3_s32(a[3], a[4], a[5]), l2 = __vimin3_s32(a[3], a[4], a[5]), d2 = a[3] + a[4] + a[5] - h2 - l2;
+    const int h3 = __vimax3_s32(a[6], a[7], a[8]), l3 = __vimin3_s32(a[6], a[7], a[8]), d3 = a[6] + a[7] + a[8] - h3 - l3;
+    const int m1 = __vimax3_s32(h1, h2, h3), lh = __vimin3_s32(h1, h2, h3), mh = h1 + h2 + h3 - m1 - lh;
+    const int dmax = __vimax3_s32(d1, d2, d3), lmax = __vimax3_s32(l1, l2, l3);
+    const int m2 = max(mh, dmax);
+    const int m3 = __vimax3_s32(min(mh, dmax), lh, lmax);
+
+    const unsigned t = (eabs & static_cast<unsigned>(kOne - 1)) != 0u ? 1u : 0u;
+    const unsigned jx = (eabs - t) >> 29;
+    const bool zero = eabs == 0u;   // e == 0: no flips, no candidate
+    const int mc = jx <= 1u ? m1 : (jx <= 3u ? m2 : m3);
+    const bool big = !(fabsf(ef) < 0x1.ep31f);
+    const bool ok = !big & (jx <= 5u) & ((mc >= (1 << 27)) | zero);
+    // ok and jx >= 1 imply that ranks 1..c are real elements (keys >= 2^27): indices are 0..8
+    if (ok & (jx >= 1u)) {
         const int i1 = ~m1 & 15;   // = 15 - (m1 & 15)
         cb[i1] = static_cast<unsigned char>(cb[i1] - sgn);
     }
-    if (ok & (j >= 3)) {
+    if (ok & (jx >= 3u)) {
         const int i2 = ~m2 & 15;
         cb[i2] = static_cast<unsigned char>(cb[i2] - sgn);
     }
-    if (ok & (j == 5)) {
+    if (ok & (jx == 5u)) {
         const int i3 = ~m3 & 15;
         cb[i3] = static_cast<unsigned char>(cb[i3] - sgn);
     }
-    // candidate: Over (j odd) -> the k-th (last flipped), Under -> the (k+1)-th
-    const int mc = (j <= 1) ? m1 : ((j <= 3) ? m2 : m3);
-    const int idx = ~mc & 15;   // at most 15: stays inside the staged channel
-    unsigned tb;
-    float Pcf;
-    squant_e_fastf(wk[idx], y, s2, tb, Pcf);   // exact value of the candidate's perturbation
-    const int Pc = __float2int_rn(__fmul_rn(Pcf, sgn_f));
-    const int vs = (j & 1) ? Pc - kOne : Pc;
-    const unsigned k = static_cast<unsigned>(j + 1) >> 1;
+    const int vs = (mc & ~15) - static_cast<int>((jx & 1u) << 30);   // Over: value after the flip
+    const unsigned k = (jx + 1u) >> 1;
     e_out = sgn * static_cast<int>(eabs - (k << 30));
     v_out = zero ? 0 : sgn * vs;
-    idx_out = idx;
+    idx_out = static_cast<unsigned>(~mc & 15);
     return !ok;
 }
 
@@ -561,6 +559,7 @@ __device__ __forceinline__ float stage_channel(const LayerDesc &L, int m, const 
         for (int i = G.t; i < kHistBins; i += G.g) hist[i] = 0;
         if (G.t == 0) {
             reinterpret_cast<int *>(red + 128)[5] = 0;                    // boundary-list count
+            reinterpret_cast<int *>(red + 128)[6] = 0;                    // redo-list count (3x3 fast path)
             *reinterpret_cast<unsigned long long *>(red + 208) = 0ull;   // channel-sum accumulator
             *reinterpret_cast<unsigned *>(red + 216) = 0u;               // absmax slot
         }
@@ -812,6 +811,7 @@ __device__ __forceinline__ void channel_body_ec(const LayerDesc &L, int m, const
 }
 
 // ---------------------------------------------------------------- SQuant-C by histogram (fast paths)
+constexpr unsigned kRedoMark = 0xffu;   // element index stored for a kernel that awaits its exact redo
 constexpr int kListCap = 128;   // the boundary list lives in the histogram's 1 KB once the scan is done
 
 __device__ __forceinline__ void hist_add(int *hist, int v)
@@ -827,13 +827,13 @@ __device__ __forceinline__ void hist_add(int *hist, int v)
 template <int KT>
 __device__ __forceinline__ void finish_channel_hist(const LayerDesc &L, int m, const Group &G,
                                                     unsigned char *slice, float s, unsigned mode,
-                                                    long long esum, float *kerr)
+                                                    long long esum, float *kerr, float y, float s2)
 {
     const int N = L.N;
     unsigned char *cbuf = slice + L.off_codes;
-    const int *ev = reinterpret_cast<const int *>(slice + L.off_ev);
-    const int *vv = reinterpret_cast<const int *>(slice + L.off_vv);
-    const unsigned char *vi = slice + L.off_vi;
+    int *ev = reinterpret_cast<int *>(slice + L.off_ev);
+    int *vv = reinterpret_cast<int *>(slice + L.off_vv);
+    unsigned char *vi = slice + L.off_vi;
     int *hist = reinterpret_cast<int *>(slice + L.off_hist);
     unsigned char *red = slice + L.off_red;
     int *bc = reinterpret_cast<int *>(red + 128);               // [0..3] scan result, [5] list count
@@ -844,7 +844,32 @@ __device__ __forceinline__ void finish_channel_hist(const LayerDesc &L, int m, c
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) esum += __shfl_xor_sync(kFull, esum, o);
     if ((G.t & 31) == 0) atomicAdd(acc, static_cast<unsigned long long>(esum));
-    G.sync();   // per-kernel data, histogram and channel sum visible
+    G.sync();   // per-kernel data, histogram, channel sum and redo list visible
+    if (KT == 9) {
+        // Kernels the fast selection reported: redone exactly from the staged weights, one
+        // thread per kernel.  The list holds N / 2 entries; beyond that (inputs made of ties or
+        // of weights tiny against the channel's scale) every thread redoes its own marked kernels.
+        const int cnt = bc[6];
+        if (cnt > 0) {   // group-uniform
+            const float *wbuf = reinterpret_cast<const float *>(slice);
+            const unsigned short *redo = reinterpret_cast<const unsigned short *>(vi + N);
+            const bool listed = cnt <= (N >> 1);
+            const int end = listed ? cnt : N;
+            for (int i = G.t; i < end; i += G.g) {
+                int n = i;
+                if (listed) n = redo[i];
+                else if (vi[i] != kRedoMark) continue;
+                const KernelOut o = kernel9_exact(wbuf + n * 9, y, s2, cbuf + n * 9);
+                ev[n] = o.e;
+                vv[n] = o.v;
+                vi[n] = static_cast<unsigned char>(o.idx);
+                if (kerr) kerr[n] = __fmul_rn(__int2float_rn(o.e), 0x1p-30f);
+                if (o.v != 0) hist_add(hist, o.v);
+                atomicAdd(acc, static_cast<unsigned long long>(static_cast<long long>(o.e)));
+            }
+            G.sync();
+        }
+    }
     long long ec = static_cast<long long>(*acc);
 
     // ---- SQuant-C: boundary bin of the candidate histogram
@@ -993,6 +1018,9 @@ __device__ __forceinline__ void channel_body_k9_fast(const LayerDesc &L, int m, 
     const float s2 = __fmul_rn(s, 0x1p-30f);
     const float y = __frcp_rn(s2);
     const int quads = N >> 2;
+    int *redo_cnt = reinterpret_cast<int *>(slice + L.off_red + 128) + 6;
+    unsigned short *redo = reinterpret_cast<unsigned short *>(vi + N);   // upper half of the index area
+    const int redo_cap = N >> 1;
     long long esum = 0;
     for (int Q = G.t; Q < quads; Q += G.g) {
         const float4 *src = reinterpret_cast<const float4 *>(wbuf) + Q * 9;
@@ -1009,23 +1037,26 @@ __device__ __forceinline__ void channel_body_k9_fast(const LayerDesc &L, int m, 
             dst[j] = __byte_perm(__byte_perm(t0, t1, 0x0040), __byte_perm(t2, t3, 0x0040), 0x5410);
         }
         int e4[4], v4[4];
-        unsigned i4 = 0, again = 0;
-        const float *wq = wbuf + Q * 36;
+        unsigned i4 = 0;
         unsigned char *cq = cbuf + Q * 36;
 #pragma unroll
         for (int kq = 0; kq < 4; ++kq) {
             float Pk[9];
 #pragma unroll
             for (int i = 0; i < 9; ++i) Pk[i] = P[9 * kq + i];
-            int idx;
-            if (kernel9_fast(Pk, wq + 9 * kq, y, s2, cq + 9 * kq, e4[kq], v4[kq], idx)) {
-                again |= 1u << kq;   // redone exactly below
+            unsigned idx;
+            if (kernel9_select(Pk, cq + 9 * kq, e4[kq], v4[kq], idx)) {   // rare: redone exactly later
+                const int pos = atomicAdd(redo_cnt, 1);
+                if (pos < redo_cap) redo[pos] = static_cast<unsigned short>(4 * Q + kq);
                 e4[kq] = 0;
                 v4[kq] = 0;
-                idx = 0;
+                idx = kRedoMark;
             }
-            hist_add(hist, v4[kq]);
-            i4 |= static_cast<unsigned>(idx) << (8 * kq);
+            if (v4[kq] != 0) {   // |v| < 2^30: the bin is in range
+                const int v = v4[kq];
+                atomicAdd(&hist[abs(v) >> 22], v > 0 ? 1 : 0x10000);
+            }
+            i4 |= idx << (8 * kq);
         }
         esum += static_cast<long long>(e4[0] + e4[1]) + (e4[2] + e4[3]);   // pairs fit 32 bits
         reinterpret_cast<int4 *>(ev)[Q] = make_int4(e4[0], e4[1], e4[2], e4[3]);
@@ -1040,23 +1071,8 @@ __device__ __forceinline__ void channel_body_k9_fast(const LayerDesc &L, int m, 
             if (kvec) __stcs(reinterpret_cast<float4 *>(kerr) + Q, f);
             else { kerr[4 * Q] = f.x; kerr[4 * Q + 1] = f.y; kerr[4 * Q + 2] = f.z; kerr[4 * Q + 3] = f.w; }
         }
-        if (again) {   // rare: kernels the fast selection handed back
-#pragma unroll 1
-            for (int kq = 0; kq < 4; ++kq) {
-                if (again & (1u << kq)) {
-                    const int n = 4 * Q + kq;
-                    const KernelOut o = kernel9_exact(wbuf + n * 9, y, s2, cbuf + n * 9);
-                    ev[n] = o.e;
-                    vv[n] = o.v;
-                    vi[n] = static_cast<unsigned char>(o.idx);
-                    if (kerr) kerr[n] = __fmul_rn(__int2float_rn(o.e), 0x1p-30f);
-                    hist_add(hist, o.v);
-                    esum += o.e;
-                }
-            }
-        }
     }
-    finish_channel_hist<9>(L, m, G, slice, s, mode, esum, kerr);
+    finish_channel_hist<9>(L, m, G, slice, s, mode, esum, kerr, y, s2);
 }
 
 // ---------------------------------------------------------------- channel body, 1x1 fast path
@@ -1105,7 +1121,7 @@ __device__ __forceinline__ void channel_body_k1_fast(const LayerDesc &L, int m, 
             else { kerr[4 * Q] = f.x; kerr[4 * Q + 1] = f.y; kerr[4 * Q + 2] = f.z; kerr[4 * Q + 3] = f.w; }
         }
     }
-    finish_channel_hist<1>(L, m, G, slice, s, mode, esum, kerr);
+    finish_channel_hist<1>(L, m, G, slice, s, mode, esum, kerr, y, s2);
 }
 
 // ---------------------------------------------------------------- self-check of the fast division
