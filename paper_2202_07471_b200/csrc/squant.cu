@@ -189,6 +189,8 @@ int build_param_plan(const squant_layer *layers, int32_t n_layers, const squant_
         sq::LaunchTable &t = p.tables.back();
         std::memset(&t, 0, sizeof(t));
         t.n_layers = n;
+        t.top_step = 0;
+        for (int st = 1; st < n; st <<= 1) t.top_step = st;
         int items = 0;
         for (int j = 0; j < n; ++j) {
             const LayerDesc &d = descs[order[base + j]];

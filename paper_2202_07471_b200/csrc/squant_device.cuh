@@ -50,7 +50,7 @@ struct Item {
 constexpr int kMaxParamLayers = 96;
 struct LaunchTable {
     int n_layers;
-    int pad;
+    int top_step;   // largest power of two below n_layers (0 for one layer): first step of the layer search
     int first_item[kMaxParamLayers + 1];
     LayerDesc layers[kMaxParamLayers];
 };
@@ -376,6 +376,7 @@ __device__ __forceinline__ int select_threshold(const Group &G, const int *vv, i
 //     qX = t - kMagic     = code * 2^30, exactly
 //     P  = cvt.rni(qX - X)   the perturbation in 2^-30 units (the difference is exact)
 // and the low byte of t's bit pattern is the code in two's complement.
+constexpr unsigned kRedoMark = 0xffu;   // element index stored for a kernel that awaits its exact redo
 constexpr float kMagic = 0x1.8p53f;   // 1.5 * 2^53: mantissa field 0x400000, low byte 0
 
 __device__ __forceinline__ float div_scaled(float w, float y, float s2)
@@ -399,6 +400,34 @@ __device__ __forceinline__ void squant_e_fast(float w, float y, float s2, unsign
     float Pf;
     squant_e_fastf(w, y, s2, tbits, Pf);
     P = __float2int_rn(Pf);
+}
+
+// The same on two weights at once with sm_100's packed fp32x2 arithmetic: each instruction
+// yields two IEEE round-to-nearest results, identical to the scalar sequence above, for one
+// issue slot.  E2 holds the channel's constants as pairs.
+struct E2 {
+    float2 y, ns2, magic, nmagic, neg1;
+};
+
+__device__ __forceinline__ E2 make_e2(float y, float s2)
+{
+    E2 c;
+    c.y = make_float2(y, y);
+    c.ns2 = make_float2(-s2, -s2);
+    c.magic = make_float2(kMagic, kMagic);
+    c.nmagic = make_float2(-kMagic, -kMagic);
+    c.neg1 = make_float2(-1.0f, -1.0f);
+    return c;
+}
+
+__device__ __forceinline__ void squant_e_fast2(float2 w, const E2 &c, float2 &t, float2 &Pf)
+{
+    const float2 x0 = __fmul2_rn(w, c.y);
+    const float2 r = __ffma2_rn(x0, c.ns2, w);      // w - x0 * s2, exact
+    const float2 X = __ffma2_rn(r, c.y, x0);        // RN(w / s2)
+    t = __fadd2_rn(X, c.magic);
+    const float2 qX = __fadd2_rn(t, c.nmagic);
+    Pf = __ffma2_rn(X, c.neg1, qX);                 // qX - X, exact
 }
 
 // Exact SQuant-K + Algorithm 3 on one 3x3 kernel from its weights in shared memory; codes are
@@ -485,19 +514,16 @@ __device__ __noinline__ KernelOut kernel9_exact(const float *wk, float y, float 
 // so is the candidate's value (the key without its index bits); otherwise the kernel is
 // reported.  The three largest keys come from a 3x3 sorting tableau: sort each triple, then
 // the column of maxima; the top three of nine lie in row 1 and column 1 (21 operations).
-__device__ __forceinline__ bool kernel9_select(const float (&Pf)[9], unsigned char *cb, int &e_out,
-                                               int &v_out, unsigned &idx_out)
+__device__ __forceinline__ bool kernel9_select(const float (&Psf)[9], float ef, unsigned char *cb,
+                                               int &e_out, int &v_out, unsigned &idx_out)
 {
-    const float ef = __fadd_rn(__fadd_rn(__fadd_rn(__fadd_rn(Pf[0], Pf[1]), __fadd_rn(Pf[2], Pf[3])),
-                                         __fadd_rn(__fadd_rn(Pf[4], Pf[5]), __fadd_rn(Pf[6], Pf[7]))),
-                               Pf[8]);
-    const float sgn_f = copysignf(1.0f, ef);
+    // Psf[i] = Pf[i] * copysign(1, ef): the perturbations normalised to the sign of the float sum
     const int sgn = (__float_as_int(ef) >> 31) | 1;
     int a[9];
     unsigned eabs = 0;   // |e| mod 2^32
 #pragma unroll
     for (int i = 0; i < 9; ++i) {
-        const int Ps = __float2int_rn(__fmul_rn(Pf[i], sgn_f));
+        const int Ps = __float2int_rn(Psf[i]);
         eabs += static_cast<unsigned>(Ps);
         a[i] = (Ps & ~15) | (15 - i);
     }
@@ -516,24 +542,24 @@ __device__ __forceinline__ bool kernel9_select(const float (&Pf)[9], unsigned ch
     const int mc = jx <= 1u ? m1 : (jx <= 3u ? m2 : m3);
     const bool big = !(fabsf(ef) < 0x1.ep31f);
     const bool ok = !big & (jx <= 5u) & ((mc >= (1 << 27)) | zero);
-    // ok and jx >= 1 imply that ranks 1..c are real elements (keys >= 2^27): indices are 0..8
-    if (ok & (jx >= 1u)) {
-        const int i1 = ~m1 & 15;   // = 15 - (m1 & 15)
-        cb[i1] = static_cast<unsigned char>(cb[i1] - sgn);
-    }
-    if (ok & (jx >= 3u)) {
-        const int i2 = ~m2 & 15;
-        cb[i2] = static_cast<unsigned char>(cb[i2] - sgn);
+    // Every key carries the index of a real element, so the positions below are 0..8 whatever
+    // the input; ranks 1 and 2 are read-modify-written unconditionally (a zero change when the
+    // flip does not apply), rank 3 is rare enough for a branch.
+    {
+        unsigned char *p1 = cb + (~m1 & 15);
+        *p1 = static_cast<unsigned char>(*p1 - ((ok & (jx >= 1u)) ? sgn : 0));
+        unsigned char *p2 = cb + (~m2 & 15);
+        *p2 = static_cast<unsigned char>(*p2 - ((ok & (jx >= 3u)) ? sgn : 0));
     }
     if (ok & (jx == 5u)) {
-        const int i3 = ~m3 & 15;
-        cb[i3] = static_cast<unsigned char>(cb[i3] - sgn);
+        unsigned char *p3 = cb + (~m3 & 15);
+        *p3 = static_cast<unsigned char>(*p3 - sgn);
     }
     const int vs = (mc & ~15) - static_cast<int>((jx & 1u) << 30);   // Over: value after the flip
     const unsigned k = (jx + 1u) >> 1;
-    e_out = sgn * static_cast<int>(eabs - (k << 30));
-    v_out = zero ? 0 : sgn * vs;
-    idx_out = static_cast<unsigned>(~mc & 15);
+    e_out = ok ? sgn * static_cast<int>(eabs - (k << 30)) : 0;
+    v_out = (ok & !zero) ? sgn * vs : 0;
+    idx_out = ok ? static_cast<unsigned>(~mc & 15) : kRedoMark;
     return !ok;
 }
 
@@ -565,15 +591,15 @@ __device__ __forceinline__ float stage_channel(const LayerDesc &L, int m, const 
         }
     }
     if ((reinterpret_cast<uintptr_t>(wg) & 15) == 0 && (NK & 3) == 0) {
-        if (G.t == 0) {
-            *flag = 0;
+        if (G.t == 0) {   // one thread waits for the copy; the others wait for it at the barrier
             mbar_init(bar, 1);
             bulk_load(wbuf, wg, static_cast<unsigned>(NK) * 4u, bar);
+            *flag = mbar_wait(bar, 0) ? 0 : 1;
         }
-        G.sync();   // barrier initialised before anyone polls it
-        if (!mbar_wait(bar, 0)) *flag = 1;
+        G.sync();   // the staged channel (written by the async proxy, observed through the mbarrier) is visible
         const int nv = NK >> 2;
         const float4 *src = reinterpret_cast<const float4 *>(wbuf);
+#pragma unroll 3
         for (int i = G.t; i < nv; i += G.g) {
             const float4 t = src[i];
             amax = fmaxf(fmaxf(amax, fabsf(t.x)), fmaxf(fabsf(t.y), fmaxf(fabsf(t.z), fabsf(t.w))));
@@ -811,7 +837,6 @@ __device__ __forceinline__ void channel_body_ec(const LayerDesc &L, int m, const
 }
 
 // ---------------------------------------------------------------- SQuant-C by histogram (fast paths)
-constexpr unsigned kRedoMark = 0xffu;   // element index stored for a kernel that awaits its exact redo
 constexpr int kListCap = 128;   // the boundary list lives in the histogram's 1 KB once the scan is done
 
 __device__ __forceinline__ void hist_add(int *hist, int v)
@@ -840,10 +865,14 @@ __device__ __forceinline__ void finish_channel_hist(const LayerDesc &L, int m, c
     unsigned long long *acc = reinterpret_cast<unsigned long long *>(red + 208);
     int2 *blist = reinterpret_cast<int2 *>(slice + L.off_hist); // boundary list: reuses the histogram after the scan
     const int quads = N >> 2;
-    // channel sum: warp shuffle, then one shared atomic per warp
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) esum += __shfl_xor_sync(kFull, esum, o);
-    if ((G.t & 31) == 0) atomicAdd(acc, static_cast<unsigned long long>(esum));
+    // channel sum: two 32-bit warp reductions (|esum| < 2^40 per thread, so the halves cannot
+    // overflow over 32 lanes), then one shared atomic per warp
+    {
+        const int hi = __reduce_add_sync(kFull, static_cast<int>(esum >> 16));
+        const int lo = __reduce_add_sync(kFull, static_cast<int>(esum & 0xffff));
+        if ((G.t & 31) == 0)
+            atomicAdd(acc, static_cast<unsigned long long>((static_cast<long long>(hi) << 16) + lo));
+    }
     G.sync();   // per-kernel data, histogram, channel sum and redo list visible
     if (KT == 9) {
         // Kernels the fast selection reported: redone exactly from the staged weights, one
@@ -942,6 +971,7 @@ __device__ __forceinline__ void finish_channel_hist(const LayerDesc &L, int m, c
         for (int Q = G.t; Q < quads; Q += G.g) {
             const int4 v4 = reinterpret_cast<const int4 *>(vv)[Q];
             const int v[4] = {v4.x, v4.y, v4.z, v4.w};
+            if (max(max(v[0] * sgn_c, v[1] * sgn_c), max(v[2] * sgn_c, v[3] * sgn_c)) < t_min) continue;
 #pragma unroll
             for (int kq = 0; kq < 4; ++kq) {
                 const int a = v[kq] * sgn_c;
@@ -1022,19 +1052,46 @@ __device__ __forceinline__ void channel_body_k9_fast(const LayerDesc &L, int m, 
     unsigned short *redo = reinterpret_cast<unsigned short *>(vi + N);   // upper half of the index area
     const int redo_cap = N >> 1;
     long long esum = 0;
+    const E2 c2 = make_e2(y, s2);
     for (int Q = G.t; Q < quads; Q += G.g) {
         const float4 *src = reinterpret_cast<const float4 *>(wbuf) + Q * 9;
         unsigned *dst = reinterpret_cast<unsigned *>(cbuf) + Q * 9;
-        float P[36];
+        float2 P2[18];   // the quad's 36 perturbations, pair p = elements 2p, 2p + 1
 #pragma unroll
         for (int j = 0; j < 9; ++j) {
             const float4 w = src[j];
-            unsigned t0, t1, t2, t3;
-            squant_e_fastf(w.x, y, s2, t0, P[4 * j]);
-            squant_e_fastf(w.y, y, s2, t1, P[4 * j + 1]);
-            squant_e_fastf(w.z, y, s2, t2, P[4 * j + 2]);
-            squant_e_fastf(w.w, y, s2, t3, P[4 * j + 3]);
-            dst[j] = __byte_perm(__byte_perm(t0, t1, 0x0040), __byte_perm(t2, t3, 0x0040), 0x5410);
+            float2 ta, tb;
+            squant_e_fast2(make_float2(w.x, w.y), c2, ta, P2[2 * j]);
+            squant_e_fast2(make_float2(w.z, w.w), c2, tb, P2[2 * j + 1]);
+            dst[j] = __byte_perm(__byte_perm(__float_as_uint(ta.x), __float_as_uint(ta.y), 0x0040),
+                                 __byte_perm(__float_as_uint(tb.x), __float_as_uint(tb.y), 0x0040), 0x5410);
+        }
+        // float sums of the four kernels (elements 0-8, 9-17, 18-26, 27-35), for their signs
+        float ef[4];
+        {
+            const float2 s0 = __fadd2_rn(__fadd2_rn(P2[0], P2[1]), __fadd2_rn(P2[2], P2[3]));
+            const float2 s1 = __fadd2_rn(__fadd2_rn(P2[5], P2[6]), __fadd2_rn(P2[7], P2[8]));
+            const float2 s2p = __fadd2_rn(__fadd2_rn(P2[9], P2[10]), __fadd2_rn(P2[11], P2[12]));
+            const float2 s3 = __fadd2_rn(__fadd2_rn(P2[14], P2[15]), __fadd2_rn(P2[16], P2[17]));
+            ef[0] = __fadd_rn(__fadd_rn(s0.x, s0.y), P2[4].x);
+            ef[1] = __fadd_rn(__fadd_rn(s1.x, s1.y), P2[4].y);
+            ef[2] = __fadd_rn(__fadd_rn(s2p.x, s2p.y), P2[13].x);
+            ef[3] = __fadd_rn(__fadd_rn(s3.x, s3.y), P2[13].y);
+        }
+        // normalise every perturbation to the sign of its kernel's sum (pairs 4 and 13 straddle two kernels)
+        {
+            const float g0 = copysignf(1.0f, ef[0]), g1 = copysignf(1.0f, ef[1]);
+            const float g2 = copysignf(1.0f, ef[2]), g3 = copysignf(1.0f, ef[3]);
+            const float2 G0 = make_float2(g0, g0), G1 = make_float2(g1, g1), G2 = make_float2(g2, g2), G3 = make_float2(g3, g3);
+#pragma unroll
+            for (int p = 0; p < 4; ++p) {
+                P2[p] = __fmul2_rn(P2[p], G0);
+                P2[5 + p] = __fmul2_rn(P2[5 + p], G1);
+                P2[9 + p] = __fmul2_rn(P2[9 + p], G2);
+                P2[14 + p] = __fmul2_rn(P2[14 + p], G3);
+            }
+            P2[4] = __fmul2_rn(P2[4], make_float2(g0, g1));
+            P2[13] = __fmul2_rn(P2[13], make_float2(g2, g3));
         }
         int e4[4], v4[4];
         unsigned i4 = 0;
@@ -1043,18 +1100,18 @@ __device__ __forceinline__ void channel_body_k9_fast(const LayerDesc &L, int m, 
         for (int kq = 0; kq < 4; ++kq) {
             float Pk[9];
 #pragma unroll
-            for (int i = 0; i < 9; ++i) Pk[i] = P[9 * kq + i];
+            for (int i = 0; i < 9; ++i) {
+                const int el = 9 * kq + i;
+                Pk[i] = (el & 1) ? P2[el >> 1].y : P2[el >> 1].x;
+            }
             unsigned idx;
-            if (kernel9_select(Pk, cq + 9 * kq, e4[kq], v4[kq], idx)) {   // rare: redone exactly later
+            if (kernel9_select(Pk, ef[kq], cq + 9 * kq, e4[kq], v4[kq], idx)) {   // rare: redone exactly later
                 const int pos = atomicAdd(redo_cnt, 1);
                 if (pos < redo_cap) redo[pos] = static_cast<unsigned short>(4 * Q + kq);
-                e4[kq] = 0;
-                v4[kq] = 0;
-                idx = kRedoMark;
             }
-            if (v4[kq] != 0) {   // |v| < 2^30: the bin is in range
+            {   // candidate histogram; |v| < 2^30, so the bin is in range (v = 0 adds nothing)
                 const int v = v4[kq];
-                atomicAdd(&hist[abs(v) >> 22], v > 0 ? 1 : 0x10000);
+                atomicAdd(&hist[abs(v) >> 22], v > 0 ? 1 : ((v >> 31) & 0x10000));
             }
             i4 |= idx << (8 * kq);
         }
@@ -1127,8 +1184,9 @@ __device__ __forceinline__ void channel_body_k1_fast(const LayerDesc &L, int m, 
 // ---------------------------------------------------------------- self-check of the fast division
 // For each given scale s (in the fast path's range) and EVERY fp32 bit pattern w with
 // |w| <= s * qmax * (1 + 2^-20) - a superset of what a channel with that scale can contain -
-// compares code and integer perturbation from the reciprocal-based SQuant-E with those from the
-// plain IEEE division.  mismatches[i] counts the disagreements for scales[i].
+// compares code and integer perturbation from the reciprocal-based SQuant-E, in its scalar and in
+// its packed fp32x2 form, with those from the plain IEEE division.  mismatches[i] counts the
+// disagreements for scales[i].
 __global__ void selfcheck_division_kernel(const float *scales, int n, int qmax,
                                           unsigned long long *mismatches)
 {
@@ -1138,19 +1196,27 @@ __global__ void selfcheck_division_kernel(const float *scales, int n, int qmax,
     const float s2 = __fmul_rn(s, 0x1p-30f);
     const float y = __frcp_rn(s2);
     const float lim = __fmul_rn(__fmul_rn(s, static_cast<float>(qmax)), 1.000001f);
+    const E2 c2 = make_e2(y, s2);
     unsigned long long bad = 0;
-    const unsigned long long total = 1ull << 32;
-    for (unsigned long long b = blockIdx.x * static_cast<unsigned long long>(blockDim.x) + threadIdx.x; b < total;
+    const unsigned long long half = 1ull << 31;   // a pair = (w, -w): both lanes of the packed sequence
+    for (unsigned long long b = blockIdx.x * static_cast<unsigned long long>(blockDim.x) + threadIdx.x; b < half;
          b += static_cast<unsigned long long>(gridDim.x) * blockDim.x) {
         const float w = __uint_as_float(static_cast<unsigned>(b));
-        if (!(fabsf(w) <= lim)) continue;   // also skips NaN
-        unsigned tb;
-        int Pf_fast;
-        squant_e_fast(w, y, s2, tb, Pf_fast);
-        int q, P;
-        squant_e(w, s, q, P);
-        const int qf = static_cast<int>(static_cast<signed char>(tb & 255u));
-        bad += (qf != q) | (Pf_fast != P);
+        if (!(w <= lim)) continue;   // also skips NaN
+        const float wp[2] = {w, -w};
+        float2 t2, P2;
+        squant_e_fast2(make_float2(wp[0], wp[1]), c2, t2, P2);
+        const float tl[2] = {t2.x, t2.y}, Pl[2] = {P2.x, P2.y};
+#pragma unroll
+        for (int l = 0; l < 2; ++l) {
+            unsigned tb;
+            int P_fast, q, P;
+            squant_e_fast(wp[l], y, s2, tb, P_fast);   // the scalar sequence (used by the exact redo)
+            squant_e(wp[l], s, q, P);                   // plain IEEE division
+            const int qs = static_cast<int>(static_cast<signed char>(tb & 255u));
+            const int qp = static_cast<int>(static_cast<signed char>(__float_as_uint(tl[l]) & 255u));
+            bad += (qs != q) | (P_fast != P) | (qp != q) | (__float2int_rn(Pl[l]) != P);
+        }
     }
     for (int o = 16; o > 0; o >>= 1) bad += __shfl_xor_sync(kFull, bad, o);
     if ((threadIdx.x & 31) == 0 && bad) atomicAdd(mismatches + si, bad);
@@ -1199,7 +1265,7 @@ squant_model_kernel(const __grid_constant__ LaunchTable tbl, int qmax, unsigned 
     const int item = blockIdx.x;
     int layer = 0;   // uniform binary search for the last layer whose first item is <= item
 #pragma unroll 1
-    for (int step = 64; step > 0; step >>= 1)
+    for (int step = tbl.top_step; step > 0; step >>= 1)
         if (layer + step < tbl.n_layers && tbl.first_item[layer + step] <= item) layer += step;
     const LayerDesc &L = tbl.layers[layer];
     const int ch0 = (item - tbl.first_item[layer]) * (kCtaThreads >> L.g_shift);
