@@ -7,7 +7,7 @@ import oracle
 import paper_2202_07471_b200 as sq
 from paper_2202_07471_b200 import workloads as W
 
-from cases import SWEEP_SHAPES, adversarial_layer, coarse
+from cases import SWEEP_SHAPES, adversarial_layer, coarse, redo_layer
 
 pytestmark = pytest.mark.gpu
 
@@ -97,6 +97,18 @@ def test_coarse_grid_ties_large_channel():
     w[:, 0, 0, 0] = 1.0
     (b,) = run_gpu([w], 8, EKC)
     assert_layer_equal(b, w, 8, EKC)
+
+
+@pytest.mark.parametrize("bits", [4, 8])
+def test_kernels_the_fast_selection_hands_back(bits):
+    """3x3 channels in which none, a few, just under half, just over half and all kernels cannot
+    be settled by the straight-line selection (tiny weights, error sums near 4): the exact redo
+    by list and by per-thread marks."""
+    ws = [redo_layer(2048, bits), redo_layer(64, bits, seed=4), redo_layer(8, bits, seed=5)]
+    for mode in (EKC, EK):
+        bufs = run_gpu(ws, bits, mode)
+        for i, (b, w) in enumerate(zip(bufs, ws)):
+            assert_layer_equal(b, w, bits, mode, tag=f"redo layer {i} mode{mode}")
 
 
 @pytest.mark.parametrize("name,bits", [("resnet18", 4), ("resnet50", 4), ("resnet50", 6), ("mobilenetv2", 4),
