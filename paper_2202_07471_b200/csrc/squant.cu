@@ -13,6 +13,7 @@
 #include <vector>
 
 #include "squant_device.cuh"
+#include "squant_pipe.cuh"
 
 namespace {
 
@@ -153,11 +154,27 @@ int build_plan(const squant_layer *layers, int32_t n_layers, const squant_option
 // CTAs (heaviest first, so the tail of the launch is made of light CTAs), at most
 // kMaxParamLayers per launch.
 struct ParamPlan {
-    std::vector<sq::LaunchTable> tables;
+    std::vector<sq::LaunchTable> tables;   // grouped kernel: one CTA per item
     std::vector<int> grids;
     int smem_bytes = 0, qmax = 0;
     unsigned mode = 0;
+    // pipelined kernel (layers of long 3x3 channels): one item per output channel
+    std::vector<sq::LaunchTable> pipe_tables;
+    std::vector<int> pipe_items, pipe_set_stride, pipe_slot;
 };
+
+int g_next_slot = 0;   // next work-counter slot of the pipelined kernel; guarded by g_mutex
+
+// Layers the pipelined kernel takes: 3x3, more than 8192 weights per output channel (the grouped
+// kernel gives such a channel a whole CTA), input channels a multiple of four, SQuant-K on, plain
+// int8 codes, and two buffer sets fit the shared memory of one SM.
+bool pipe_eligible(const squant_layer &l, const LayerDesc &d, const squant_options &o, int max_smem)
+{
+    if (d.K != 9 || (d.N & 3) != 0 || d.NK <= 8192 || d.g != sq::kCtaThreads) return false;
+    if (!(o.mode & SQUANT_MODE_K) || (o.flags & SQUANT_FLAG_PACK_INT4) || l.dequant) return false;
+    if ((reinterpret_cast<uintptr_t>(l.w) & 15) || (reinterpret_cast<uintptr_t>(l.codes) & 15)) return false;
+    return 2 * d.slice_bytes + sq::kPipeCtrlBytes <= max_smem;
+}
 
 int build_param_plan(const squant_layer *layers, int32_t n_layers, const squant_options &o,
                      int max_smem, ParamPlan &p)
@@ -166,13 +183,39 @@ int build_param_plan(const squant_layer *layers, int32_t n_layers, const squant_
     p.mode = o.mode | ((o.flags & SQUANT_FLAG_PACK_INT4) ? sq::kModePackInt4 : 0u);
     p.smem_bytes = 0;
     std::vector<LayerDesc> descs(n_layers);
-    std::vector<int> order(n_layers);
+    std::vector<int> order, piped;
     for (int i = 0; i < n_layers; ++i) {
         const int64_t cta_smem = layout_layer(layers[i], descs[i], o.mode);
         if (cta_smem > max_smem) return SQUANT_ERR_TOO_WIDE;
+        if (pipe_eligible(layers[i], descs[i], o, max_smem)) {
+            piped.push_back(i);
+            continue;
+        }
         if (cta_smem > p.smem_bytes) p.smem_bytes = static_cast<int>(cta_smem);
-        order[i] = i;
+        order.push_back(i);
     }
+    for (size_t base = 0; base < piped.size(); base += sq::kMaxParamLayers) {
+        const int n = static_cast<int>(std::min<size_t>(piped.size() - base, sq::kMaxParamLayers));
+        p.pipe_tables.emplace_back();
+        sq::LaunchTable &t = p.pipe_tables.back();
+        std::memset(&t, 0, sizeof(t));
+        t.n_layers = n;
+        for (int st = 1; st < n; st <<= 1) t.top_step = st;
+        int items = 0, stride = 0;
+        for (int j = 0; j < n; ++j) {
+            const LayerDesc &d = descs[piped[base + j]];
+            t.layers[j] = d;
+            t.first_item[j] = items;
+            items += d.M;
+            stride = std::max(stride, d.slice_bytes);
+        }
+        for (int j = n; j <= sq::kMaxParamLayers; ++j) t.first_item[j] = items;
+        p.pipe_items.push_back(items);
+        p.pipe_set_stride.push_back(stride);
+        p.pipe_slot.push_back(g_next_slot);
+        g_next_slot = (g_next_slot + 1) % sq::kTicketSlots;
+    }
+    n_layers = static_cast<int32_t>(order.size());   // the grouped kernel takes the rest
     // Estimated duration of one CTA of the layer.  Kernel sizes other than 1x1 and 3x3 take the
     // general per-thread path, which is latency-bound and far slower per weight (a 7x7 stem CTA
     // is the longest of a whole ResNet), so those start first.
@@ -215,6 +258,7 @@ struct CachedPlan {
 
 std::list<CachedPlan> g_plans;              // most recently used first
 std::vector<int> g_smem_limit_by_device;   // opt-in limit set on the kernels, per device
+std::vector<int> g_sm_count_by_device;     // multiprocessors, per device
 
 std::string plan_key(const squant_layer *layers, int32_t n_layers, const squant_options &o)
 {
@@ -234,6 +278,12 @@ int device_smem_limit(int device, int &limit)
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, v));
         SQ_CUDA(cudaFuncSetAttribute(sq::squant_table_kernel,
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, v));
+        SQ_CUDA(cudaFuncSetAttribute(sq::squant_pipe_kernel,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, v));
+        int sms = 0;
+        SQ_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
+        if (static_cast<int>(g_sm_count_by_device.size()) <= device) g_sm_count_by_device.resize(device + 1, 0);
+        g_sm_count_by_device[device] = sms;
         g_smem_limit_by_device[device] = v;
     }
     limit = g_smem_limit_by_device[device];
@@ -268,6 +318,18 @@ int get_plan(const squant_layer *layers, int32_t n_layers, const squant_options 
 
 int launch_plan(const ParamPlan &p, cudaStream_t stream)
 {
+    // long 3x3 channels first: one persistent CTA per multiprocessor
+    for (size_t c = 0; c < p.pipe_tables.size(); ++c) {
+        if (p.pipe_items[c] == 0) continue;
+        int device = 0;
+        SQ_CUDA(cudaGetDevice(&device));
+        const int grid = std::min(p.pipe_items[c], std::max(g_sm_count_by_device[device], 1));
+        const int smem = 2 * p.pipe_set_stride[c] + sq::kPipeCtrlBytes;
+        sq::squant_pipe_kernel<<<grid, sq::kPipeThreads, smem, stream>>>(p.pipe_tables[c], p.qmax, p.mode, p.pipe_items[c],
+                                                                     p.pipe_slot[c], p.pipe_set_stride[c]);
+        SQ_CUDA(cudaGetLastError());
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+    }
     for (size_t c = 0; c < p.tables.size(); ++c) {
         if (p.grids[c] == 0) continue;
         sq::squant_model_kernel<<<p.grids[c], sq::kCtaThreads, p.smem_bytes, stream>>>(p.tables[c], p.qmax, p.mode);

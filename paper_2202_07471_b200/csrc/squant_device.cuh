@@ -93,6 +93,13 @@ __device__ __forceinline__ void bulk_load(void *dst, const void *src, unsigned b
                  : "memory");
 }
 
+// One arrival on `bar` (release semantics: the thread's earlier writes are visible to a thread
+// that observes the phase completing).
+__device__ __forceinline__ void mbar_arrive(void *bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+
 // Bounded wait for phase `parity` of `bar`.  False if the limit ran out.
 __device__ __forceinline__ bool mbar_wait(void *bar, unsigned parity)
 {
@@ -437,15 +444,22 @@ struct KernelOut {
     int e, v, idx;
 };
 
-__device__ __noinline__ KernelOut kernel9_exact(const float *wk, float y, float s2, unsigned char *cb)
+// kDiv = false: SQuant-E by the reciprocal sequence (y, s2 as in squant_e_fast); kDiv = true: by
+// the plain IEEE division, for scales outside the reciprocal's range (y is the scale s then).
+template <bool kDiv>
+__device__ __noinline__ KernelOut kernel9_exact_t(const float *wk, float y, float s2, unsigned char *cb)
 {
     int P[9], q[9];
     long long e = 0;
 #pragma unroll
     for (int i = 0; i < 9; ++i) {
-        unsigned tb;
-        squant_e_fast(wk[i], y, s2, tb, P[i]);
-        q[i] = static_cast<int>(tb & 255u);
+        if (kDiv) {
+            squant_e(wk[i], y, q[i], P[i]);
+        } else {
+            unsigned tb;
+            squant_e_fast(wk[i], y, s2, tb, P[i]);
+            q[i] = static_cast<int>(tb & 255u);
+        }
         e += P[i];
     }
     int v = 0, idx = 0;
@@ -488,6 +502,11 @@ __device__ __noinline__ KernelOut kernel9_exact(const float *wk, float y, float 
     o.v = v;
     o.idx = idx;
     return o;
+}
+
+__device__ __forceinline__ KernelOut kernel9_exact(const float *wk, float y, float s2, unsigned char *cb)
+{
+    return kernel9_exact_t<false>(wk, y, s2, cb);
 }
 
 // Fast SQuant-K + Algorithm 3 on one 3x3 kernel whose exact perturbations Pf[0..8] (floats, in
@@ -852,7 +871,8 @@ __device__ __forceinline__ void hist_add(int *hist, int v)
 template <int KT>
 __device__ __forceinline__ void finish_channel_hist(const LayerDesc &L, int m, const Group &G,
                                                     unsigned char *slice, float s, unsigned mode,
-                                                    long long esum, float *kerr, float y, float s2)
+                                                    long long esum, float *kerr, float y, float s2,
+                                                    void *w_release = nullptr)
 {
     const int N = L.N;
     unsigned char *cbuf = slice + L.off_codes;
@@ -898,6 +918,8 @@ __device__ __forceinline__ void finish_channel_hist(const LayerDesc &L, int m, c
             }
             G.sync();
         }
+        // the staged weights are dead from here on: a pipelined caller lets the next copy start
+        if (w_release != nullptr && G.t == 0) mbar_arrive(w_release);
     }
     long long ec = static_cast<long long>(*acc);
 
@@ -1032,8 +1054,8 @@ __device__ __forceinline__ void finish_channel_hist(const LayerDesc &L, int m, c
 // kernels above it are flipped, the few inside it are collected in a list and ranked exactly
 // (|v| descending, kernel index ascending).  A boundary bin too crowded for the list (massive
 // ties) falls back to the general radix select.
-__device__ __forceinline__ void channel_body_k9_fast(const LayerDesc &L, int m, const Group &G,
-                                                     unsigned char *slice, float s, unsigned mode)
+__device__ __forceinline__ long long k9_quantize(const LayerDesc &L, int m, const Group &G,
+                                                 unsigned char *slice, float s, float s2, float y)
 {
     const int N = L.N;
     const float *wbuf = reinterpret_cast<const float *>(slice);
@@ -1045,8 +1067,7 @@ __device__ __forceinline__ void channel_body_k9_fast(const LayerDesc &L, int m, 
     float *kerr = L.kerr ? L.kerr + static_cast<size_t>(m) * N : nullptr;
     const bool kvec = (reinterpret_cast<uintptr_t>(kerr) & 15) == 0;
 
-    const float s2 = __fmul_rn(s, 0x1p-30f);
-    const float y = __frcp_rn(s2);
+    (void)s;
     const int quads = N >> 2;
     int *redo_cnt = reinterpret_cast<int *>(slice + L.off_red + 128) + 6;
     unsigned short *redo = reinterpret_cast<unsigned short *>(vi + N);   // upper half of the index area
@@ -1129,6 +1150,16 @@ __device__ __forceinline__ void channel_body_k9_fast(const LayerDesc &L, int m, 
             else { kerr[4 * Q] = f.x; kerr[4 * Q + 1] = f.y; kerr[4 * Q + 2] = f.z; kerr[4 * Q + 3] = f.w; }
         }
     }
+    return esum;
+}
+
+__device__ __forceinline__ void channel_body_k9_fast(const LayerDesc &L, int m, const Group &G,
+                                                     unsigned char *slice, float s, unsigned mode)
+{
+    const float s2 = __fmul_rn(s, 0x1p-30f);
+    const float y = __frcp_rn(s2);
+    const long long esum = k9_quantize(L, m, G, slice, s, s2, y);
+    float *kerr = L.kerr ? L.kerr + static_cast<size_t>(m) * L.N : nullptr;
     finish_channel_hist<9>(L, m, G, slice, s, mode, esum, kerr, y, s2);
 }
 
