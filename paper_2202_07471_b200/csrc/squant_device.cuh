@@ -523,7 +523,9 @@ __device__ __forceinline__ KernelOut kernel9_exact(const float *wk, float y, flo
 // i.e. floor(|e| / 2^29) with "exactly k + 1/2" falling to the lower value.  Then the flip count
 // of Algorithm 2 is k = (jx + 1) / 2, the kernel is Over SQuant iff jx is odd, and the candidate
 // of Algorithm 3 is the element of rank c = (jx + 2) / 2 (the last flipped one when Over, the
-// first un-flipped one otherwise).  jx <= 5 is handled (k <= 3, c <= 3).
+// first un-flipped one otherwise).  Every jx = 0..7 is handled (k <= 4, c <= 4); what is left for
+// the exact routine is |e| >= 3.75, uncertified keys and a wrong float sign: about one kernel in
+// 10^5 on random weights.
 //
 // Selection.  Keys are the sign-normalised integer perturbations with the element index folded
 // into their low four bits, (P & ~15) | (15 - i): distinct, and ordered like Algorithm 2's
@@ -531,8 +533,9 @@ __device__ __forceinline__ KernelOut kernel9_exact(const float *wk, float y, flo
 // every element with P >= 2^27: its quotient w/s * 2^30 is an fp32 number of magnitude >= 2^27,
 // hence a multiple of 16.  So if the key of rank c is >= 2^27 the first c ranks are exact, and
 // so is the candidate's value (the key without its index bits); otherwise the kernel is
-// reported.  The three largest keys come from a 3x3 sorting tableau: sort each triple, then
-// the column of maxima; the top three of nine lie in row 1 and column 1 (21 operations).
+// reported.  The four largest keys come from a 3x3 sorting tableau: sort each triple (rows), then
+// the columns; an entry in row i, column j has at least i * j - 1 entries above it, so the top
+// four of nine lie in row 1, column 1 and position (2, 2) (28 operations).
 __device__ __forceinline__ bool kernel9_select(const float (&Psf)[9], float ef, unsigned char *cb,
                                                int &e_out, int &v_out, unsigned &idx_out)
 {
@@ -552,27 +555,36 @@ __device__ __forceinline__ bool kernel9_select(const float (&Psf)[9], float ef, 
     const int h3 = __vimax3_s32(a[6], a[7], a[8]), l3 = __vimin3_s32(a[6], a[7], a[8]), d3 = a[6] + a[7] + a[8] - h3 - l3;
     const int m1 = __vimax3_s32(h1, h2, h3), lh = __vimin3_s32(h1, h2, h3), mh = h1 + h2 + h3 - m1 - lh;
     const int dmax = __vimax3_s32(d1, d2, d3), lmax = __vimax3_s32(l1, l2, l3);
-    const int m2 = max(mh, dmax);
-    const int m3 = __vimax3_s32(min(mh, dmax), lh, lmax);
+    const int m2 = max(mh, dmax), B = min(mh, dmax);
+    const int m3 = __vimax3_s32(B, lh, lmax);
+    // fourth: the runner-up of {B, lh, lmax} or the middle one of the triples' middle keys
+    const int dmed = d1 + d2 + d3 - dmax - __vimin3_s32(d1, d2, d3);
+    const int m4 = max(B + lh + lmax - m3 - __vimin3_s32(B, lh, lmax), dmed);
 
     const unsigned t = (eabs & static_cast<unsigned>(kOne - 1)) != 0u ? 1u : 0u;
-    const unsigned jx = (eabs - t) >> 29;
+    const unsigned jx = (eabs - t) >> 29;   // <= 7 for any 32-bit value
     const bool zero = eabs == 0u;   // e == 0: no flips, no candidate
-    const int mc = jx <= 1u ? m1 : (jx <= 3u ? m2 : m3);
-    const bool big = !(fabsf(ef) < 0x1.ep31f);
-    const bool ok = !big & (jx <= 5u) & ((mc >= (1 << 27)) | zero);
+    const int mc = jx <= 1u ? m1 : (jx <= 3u ? m2 : (jx <= 5u ? m3 : m4));
+    // |float sum| < 3.75 * 2^30 bounds the true |e| below 0xF0001000; a sum that wrapped because
+    // the float sign was wrong is >= 0xFFFFF000
+    const bool big = !(fabsf(ef) < 0x1.ep31f) | (eabs >= 0xF8000000u);
+    const bool ok = !big & ((mc >= (1 << 27)) | zero);
     // Every key carries the index of a real element, so the positions below are 0..8 whatever
     // the input; ranks 1 and 2 are read-modify-written unconditionally (a zero change when the
-    // flip does not apply), rank 3 is rare enough for a branch.
+    // flip does not apply), ranks 3 and 4 are rare enough for a branch.
     {
         unsigned char *p1 = cb + (~m1 & 15);
         *p1 = static_cast<unsigned char>(*p1 - ((ok & (jx >= 1u)) ? sgn : 0));
         unsigned char *p2 = cb + (~m2 & 15);
         *p2 = static_cast<unsigned char>(*p2 - ((ok & (jx >= 3u)) ? sgn : 0));
     }
-    if (ok & (jx == 5u)) {
+    if (ok & (jx >= 5u)) {
         unsigned char *p3 = cb + (~m3 & 15);
         *p3 = static_cast<unsigned char>(*p3 - sgn);
+        if (jx == 7u) {
+            unsigned char *p4 = cb + (~m4 & 15);
+            *p4 = static_cast<unsigned char>(*p4 - sgn);
+        }
     }
     const int vs = (mc & ~15) - static_cast<int>((jx & 1u) << 30);   // Over: value after the flip
     const unsigned k = (jx + 1u) >> 1;
