@@ -210,6 +210,10 @@ int build_param_plan(const squant_layer *layers, int32_t n_layers, const squant_
             stride = std::max(stride, d.slice_bytes);
         }
         for (int j = n; j <= sq::kMaxParamLayers; ++j) t.first_item[j] = items;
+        for (int j = 0; j < n; ++j) {   // one place for the channel-step scratch in every layer: the end of a set
+            t.layers[j].off_hist = stride - sq::kPipeScratchBytes;
+            t.layers[j].off_red = t.layers[j].off_hist + 4 * sq::kHistBins;
+        }
         p.pipe_items.push_back(items);
         p.pipe_set_stride.push_back(stride);
         p.pipe_slot.push_back(g_next_slot);

@@ -27,6 +27,7 @@ constexpr int kPipeQuantThreads = 512;
 constexpr int kPipeFinThreads = 128;
 constexpr int kPipeThreads = kPipeQuantThreads + kPipeFinThreads + 32;
 constexpr int kPipeCtrlBytes = 256;
+constexpr int kPipeScratchBytes = 4 * kHistBins + 256;   // histogram + reduction area at the end of a set
 
 // Work counters, one slot per launch plan.  Launches that share a slot must not overlap; a slot
 // belongs to one plan, i.e. to one set of output buffers, for which overlapping launches would
@@ -41,21 +42,31 @@ struct PipeCtrl {
     unsigned long long wfree[2];   // the staged weights are dead (finishers -> copy warp)
     unsigned long long qdone[2];   // codes, candidates, histogram, sums are complete (quantizers -> finishers)
     unsigned long long afree[2];   // the set's buffers may be rewritten (finishers -> quantizers)
-    int ring[2];                   // channel (item) in the set, -1: no more work
+    int ring[2];                   // channel (item) being staged into the set, -1: no more work (copy warp -> quantizers)
+    int fitem[2];                  // the same, handed on by the quantizers: the copy warp may already have
+                                   // written the set's next channel into ring[] when the finishers start
     unsigned amax[3];              // absmax accumulators, rotating
     float scale[2];                // the channel's scale, for the finishers
+    int abort;                     // a wait ran out: nobody waits any more (the launch's outputs are void)
 };
 static_assert(sizeof(PipeCtrl) <= kPipeCtrlBytes, "control block too large");
 
-__device__ __forceinline__ void pipe_wait(void *bar, unsigned parity)
+// Bounded wait.  After the first wait of the CTA that ran out, all waits return at once: the
+// kernel then runs through its remaining channels without synchronisation (every index it
+// forms is bounded whatever the data) and ends; the status word tells the host.
+__device__ __forceinline__ void pipe_wait(PipeCtrl *ctrl, void *bar, unsigned parity)
 {
-    if (!mbar_wait(bar, parity)) atomicExch(&g_device_status, 1);
+    if (*reinterpret_cast<volatile int *>(&ctrl->abort)) return;
+    if (!mbar_wait(bar, parity)) {
+        *reinterpret_cast<volatile int *>(&ctrl->abort) = 1;
+        atomicExch(&g_device_status, 1);
+    }
 }
 
 // Lane 0 of the warp waits, the others wait for lane 0.
-__device__ __forceinline__ void pipe_wait_warp(void *bar, unsigned parity)
+__device__ __forceinline__ void pipe_wait_warp(PipeCtrl *ctrl, void *bar, unsigned parity)
 {
-    if ((threadIdx.x & 31) == 0) pipe_wait(bar, parity);
+    if ((threadIdx.x & 31) == 0) pipe_wait(ctrl, bar, parity);
     __syncwarp();
 }
 
@@ -105,7 +116,14 @@ squant_pipe_kernel(const __grid_constant__ LaunchTable tbl, int qmax, unsigned m
     extern __shared__ __align__(16) unsigned char smem[];
     PipeCtrl *ctrl = reinterpret_cast<PipeCtrl *>(smem + 2 * static_cast<size_t>(set_stride));
     const int tid = threadIdx.x;
+    // In every layer of the launch the channel-step scratch (histogram, then the reduction area)
+    // is the last kPipeScratchBytes of a set: it can be cleared without knowing the layer.
+    const int hist_off = set_stride - kPipeScratchBytes, red_off = hist_off + 4 * kHistBins;
     if (tid < kPipeCtrlBytes / 4) reinterpret_cast<int *>(ctrl)[tid] = 0;
+    for (int j = tid; j < 2 * (kPipeScratchBytes / 4); j += kPipeThreads) {
+        const int b = j / (kPipeScratchBytes / 4), k = j % (kPipeScratchBytes / 4);
+        reinterpret_cast<int *>(smem + static_cast<size_t>(b) * set_stride + hist_off)[k] = 0;
+    }
     __syncthreads();
     if (tid == 0) {
         for (int b = 0; b < 2; ++b) {
@@ -127,7 +145,16 @@ squant_pipe_kernel(const __grid_constant__ LaunchTable tbl, int qmax, unsigned m
                 const unsigned t = gridDim.x + atomicAdd(&g_ticket[slot], 1u);
                 item = t < static_cast<unsigned>(n_items) ? static_cast<int>(t) : -1;
             }
-            if (u >= 1) pipe_wait(&ctrl->wfree[b], static_cast<unsigned>(u - 1) & 1u);
+            if (u >= 1) {
+                // The set's staged weights are dead once its quantizers are done, unless kernels
+                // wait for the exact redo: then the finishers say when.  (Skipping the second
+                // wait is safe: the finishers still arrive once per channel, and a later wait
+                // names the phase it needs.)
+                const unsigned par = static_cast<unsigned>(u - 1) & 1u;
+                pipe_wait(ctrl, &ctrl->qdone[b], par);
+                const int redo = reinterpret_cast<const volatile int *>(smem + static_cast<size_t>(b) * set_stride + red_off + 128)[6];
+                if (redo != 0) pipe_wait(ctrl, &ctrl->wfree[b], par);
+            }
             ctrl->ring[b] = item;
             if (item < 0) {
                 mbar_arrive(&ctrl->full[b]);
@@ -157,28 +184,20 @@ squant_pipe_kernel(const __grid_constant__ LaunchTable tbl, int qmax, unsigned m
         G.bar = 1;
         for (int i = 0;; ++i) {
             const int b = i & 1, u = i >> 1;
-            pipe_wait_warp(&ctrl->full[b], static_cast<unsigned>(u) & 1u);
+            pipe_wait_warp(ctrl, &ctrl->full[b], static_cast<unsigned>(u) & 1u);
             const int item = ctrl->ring[b];
-            if (item < 0) {
-                if ((tid & 31) == 0) mbar_arrive(&ctrl->qdone[b]);   // passes the end on to the finishers
+            if (item < 0) {   // pass the end on to the finishers (once they are done with the set's last channel)
+                if (u >= 1) pipe_wait_warp(ctrl, &ctrl->afree[b], static_cast<unsigned>(u - 1) & 1u);
+                if (tid == 0) ctrl->fitem[b] = -1;
+                G.sync();
+                if ((tid & 31) == 0) mbar_arrive(&ctrl->qdone[b]);
                 break;
             }
             const int layer = pipe_layer_of(tbl, item);
             const LayerDesc &L = tbl.layers[layer];
             const int m = item - tbl.first_item[layer];
             unsigned char *slice = smem + static_cast<size_t>(b) * set_stride;
-            if (u >= 1) pipe_wait_warp(&ctrl->afree[b], static_cast<unsigned>(u - 1) & 1u);
-            {   // channel-step scratch of the set starts at zero; the barrier below publishes it
-                int *hist = reinterpret_cast<int *>(slice + L.off_hist);
-                if (tid < kHistBins) hist[tid] = 0;
-                if (tid == 0) {
-                    unsigned char *red = slice + L.off_red;
-                    reinterpret_cast<int *>(red + 128)[5] = 0;                    // boundary-list count
-                    reinterpret_cast<int *>(red + 128)[6] = 0;                    // redo-list count
-                    *reinterpret_cast<unsigned long long *>(red + 208) = 0ull;   // channel-sum accumulator
-                    ctrl->amax[(i + 1) % 3] = 0u;   // the next channel's accumulator: idle since two barriers ago
-                }
-            }
+            if (tid == 0) ctrl->amax[(i + 1) % 3] = 0u;   // the next channel's accumulator: idle since two barriers ago
             float amax = 0.0f;
             {
                 const int nv = L.NK >> 2;
@@ -194,7 +213,12 @@ squant_pipe_kernel(const __grid_constant__ LaunchTable tbl, int qmax, unsigned m
             G.sync();
             amax = __uint_as_float(ctrl->amax[i % 3]);
             const float s = (amax < 0x1p-100f) ? 1.0f : __fdiv_rn(amax, static_cast<float>(qmax));
-            if (tid == 0) ctrl->scale[b] = s;
+            // only now are the set's other buffers needed: the finishers have cleared the scratch
+            if (u >= 1) pipe_wait_warp(ctrl, &ctrl->afree[b], static_cast<unsigned>(u - 1) & 1u);
+            if (tid == 0) {
+                ctrl->scale[b] = s;
+                ctrl->fitem[b] = item;
+            }
             long long esum;
             if (s >= 0x1p-60f && s <= 0x1p60f) {
                 const float s2 = __fmul_rn(s, 0x1p-30f);
@@ -222,8 +246,8 @@ squant_pipe_kernel(const __grid_constant__ LaunchTable tbl, int qmax, unsigned m
     G.bar = 2;
     for (int i = 0;; ++i) {
         const int b = i & 1, u = i >> 1;
-        pipe_wait_warp(&ctrl->qdone[b], static_cast<unsigned>(u) & 1u);
-        const int item = ctrl->ring[b];
+        pipe_wait_warp(ctrl, &ctrl->qdone[b], static_cast<unsigned>(u) & 1u);
+        const int item = ctrl->fitem[b];
         if (item < 0) break;
         const int layer = pipe_layer_of(tbl, item);
         const LayerDesc &L = tbl.layers[layer];
@@ -235,6 +259,17 @@ squant_pipe_kernel(const __grid_constant__ LaunchTable tbl, int qmax, unsigned m
         float *kerr = L.kerr ? L.kerr + static_cast<size_t>(m) * L.N : nullptr;
         finish_channel_hist<9>(L, m, G, slice, s, mode, 0ll, kerr, y, s2, &ctrl->wfree[b]);
         G.sync();   // every finisher is done with the set; the first one has waited for its bulk store
+        {   // leave the channel-step scratch cleared for the set's next channel
+            int *scratch = reinterpret_cast<int *>(slice + hist_off);
+            for (int j = G.t; j < kHistBins; j += kPipeFinThreads) scratch[j] = 0;
+            if (G.t == 0) {
+                unsigned char *red = slice + red_off;
+                reinterpret_cast<int *>(red + 128)[5] = 0;                    // boundary-list count
+                reinterpret_cast<int *>(red + 128)[6] = 0;                    // redo-list count
+                *reinterpret_cast<unsigned long long *>(red + 208) = 0ull;   // channel-sum accumulator
+            }
+        }
+        G.sync();
         if (G.t == 0) mbar_arrive(&ctrl->afree[b]);
     }
 }
