@@ -210,9 +210,18 @@ int build_param_plan(const squant_layer *layers, int32_t n_layers, const squant_
             stride = std::max(stride, d.slice_bytes);
         }
         for (int j = n; j <= sq::kMaxParamLayers; ++j) t.first_item[j] = items;
-        for (int j = 0; j < n; ++j) {   // one place for the channel-step scratch in every layer: the end of a set
-            t.layers[j].off_hist = stride - sq::kPipeScratchBytes;
-            t.layers[j].off_red = t.layers[j].off_hist + 4 * sq::kHistBins;
+        // One layout for every layer of the launch, that of the widest one: the staging area of a
+        // long channel must not reach into the buffers the finishers still use for a shorter one
+        // that had the set before, and the channel-step scratch is found (and cleared) without
+        // knowing the layer.  It sits at the end of a set.
+        int widest = 0;
+        for (int j = 1; j < n; ++j)
+            if (t.layers[j].slice_bytes > t.layers[widest].slice_bytes) widest = j;
+        for (int j = 0; j < n; ++j) {
+            LayerDesc &d = t.layers[j];
+            const LayerDesc &wd = t.layers[widest];
+            d.off_codes = wd.off_codes; d.off_ev = wd.off_ev; d.off_vv = wd.off_vv; d.off_vi = wd.off_vi;
+            d.off_hist = wd.off_hist; d.off_red = wd.off_red; d.slice_bytes = wd.slice_bytes;
         }
         p.pipe_items.push_back(items);
         p.pipe_set_stride.push_back(stride);

@@ -111,6 +111,27 @@ def test_kernels_the_fast_selection_hands_back(bits):
             assert_layer_equal(b, w, bits, mode, tag=f"redo layer {i} mode{mode}")
 
 
+@pytest.mark.parametrize("bits,mode", [(4, EKC), (8, EKC), (3, EK)])
+def test_long_3x3_channels_pipelined_kernel(bits, mode):
+    """Layers of long 3x3 channels (more than 8192 weights each) take the pipelined kernel: several
+    such layers of different widths in one launch (one, a few and many more channels than the GPU
+    has multiprocessors), next to layers that stay with the grouped kernel, with special channels
+    (zero, single non-zero, constant, scales far outside the reciprocal's range, ties)."""
+    shapes = [(1, 2048, 3, 3), (5, 1024, 3, 3), (333, 1000, 3, 3), (7, 1400, 3, 3), (40, 2048, 3, 3),
+              (9, 912, 3, 3), (6, 2044, 3, 3), (3, 2052, 3, 3), (4, 512, 3, 3), (11, 4100, 1, 1)]
+    ws = [adversarial_layer(s, seed=100 * bits + i) for i, s in enumerate(shapes)]
+    bufs = run_gpu(ws, bits, mode)
+    for i, (b, w) in enumerate(zip(bufs, ws)):
+        assert_layer_equal(b, w, bits, mode, tag=f"shape{shapes[i]} mode{mode}")
+    # the same buffers again: the work counter of the launch plan starts clean every time
+    for b in bufs:
+        b.codes.fill_(-128)
+    sq.squant_quantize_model(bufs, bits=bits, mode=mode)
+    sq.squant_device_status()
+    for i, (b, w) in enumerate(zip(bufs, ws)):
+        assert_layer_equal(b, w, bits, mode, tag=f"second run shape{shapes[i]}")
+
+
 @pytest.mark.parametrize("name,bits", [("resnet18", 4), ("resnet50", 4), ("resnet50", 6), ("mobilenetv2", 4),
                                        ("mixed_kernels", 4)])
 def test_model_configs_full(name, bits):
