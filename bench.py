@@ -45,7 +45,7 @@ def algorithmic_bytes(shapes) -> float:
 
 def source_digest() -> str:
     h = hashlib.sha256()
-    for f in ("squant.cu", "squant_device.cuh"):
+    for f in ("squant.cu", "squant_device.cuh", "squant_pipe.cuh"):
         with open(os.path.join(ROOT, "paper_2202_07471_b200", "csrc", f), "rb") as fh:
             h.update(fh.read())
     return h.hexdigest()[:16]
@@ -297,7 +297,7 @@ def run_cuda(args):
         "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "traffic": ncu_traffic(), "peak_kind": f"of {peak_kind}",
-                     "kernel": "squant_model_kernel", "kernel_ms": kernel_ms,
+                     "kernel": "squant_pipe_kernel", "kernel_ms": kernel_ms,
                      "algorithmic_bytes_per_launch": alg},
     }
     out.update(extra)
