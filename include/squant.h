@@ -103,8 +103,10 @@ typedef struct squant_layer {
 int squant_quantize_layer(const squant_layer *layer, const squant_options *opt, void *cuda_stream);
 
 /*
- * Algorithm 1 on every layer of a model in ONE grouped kernel launch (the paper sums
- * per-layer times and notes that layers could be quantized in parallel, Sec. 4.2).
+ * Algorithm 1 on every layer of a model in one pass (the paper sums per-layer times and notes
+ * that layers could be quantized in parallel, Sec. 4.2): ONE grouped kernel launch for all
+ * layers, plus one launch of a pipelined kernel for those layers whose 3x3 output channels are
+ * longer than 8192 weights (cin a multiple of 4 and at most 2048, SQuant-K on, int8 codes).
  *
  *   layers, n_layers  host array of descriptors holding DEVICE pointers; n_layers >= 0
  *   opt               bits / mode / flags shared by all layers; NULL means 4 bit, E|K|C, narrow
@@ -113,9 +115,12 @@ int squant_quantize_layer(const squant_layer *layer, const squant_options *opt, 
  * The launch table (layer descriptors) travels by value in the kernel's parameter space: the call
  * allocates no device memory, uploads nothing and never synchronises; more than 96 layers are
  * issued as several launches.  Host-side launch tables of recent calls are cached.  Outputs are
- * valid when the stream reaches the end of the launch.  All arguments are validated on the host
- * first; a failed call launches
- * nothing and writes nothing.  Returns SQUANT_OK or a negative SQUANT_ERR_* code.
+ * valid when the stream reaches the end of the launches.  The pipelined kernel hands out its
+ * channels through a counter in device memory that belongs to the cached launch tables of these
+ * exact descriptors: two calls with the SAME descriptors must not overlap on the GPU (they would
+ * race on the outputs anyway); calls with different descriptors may.  All arguments are validated
+ * on the host first; a failed call launches nothing and writes nothing.  Returns SQUANT_OK or a
+ * negative SQUANT_ERR_* code.
  */
 int squant_quantize_model(const squant_layer *layers, int32_t n_layers, const squant_options *opt,
                           void *cuda_stream);
@@ -130,8 +135,10 @@ int squant_quantize_model_host(const squant_layer *layers, int32_t n_layers,
                                const squant_options *opt, void *cuda_stream);
 
 /*
- * Geometry of the launch that squant_quantize_model would issue for these descriptors
- * (pointers are not dereferenced and may be NULL here).  Any output may be NULL.
+ * Geometry of the grouped launch (one thread block per 512/g output channels) that covers
+ * these descriptors, as squant_quantize_layer_noalloc issues it (pointers are not dereferenced
+ * and may be NULL here).  squant_quantize_model itself sends layers of long 3x3 channels to its
+ * pipelined kernel instead, whose grid is one block per multiprocessor.  Any output may be NULL.
  */
 int squant_plan_info(const squant_layer *layers, int32_t n_layers, const squant_options *opt,
                      int32_t *grid_ctas, int32_t *cta_threads, int32_t *dynamic_smem_bytes);
