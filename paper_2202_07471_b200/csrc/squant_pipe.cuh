@@ -210,11 +210,12 @@ squant_pipe_kernel(const __grid_constant__ LaunchTable tbl, int qmax, unsigned m
             }
             const unsigned wmax = __reduce_max_sync(kFull, __float_as_uint(amax));   // >= 0: uint order = float order
             if ((tid & 31) == 0) atomicMax(&ctrl->amax[i % 3], wmax);
+            // From here on the set's other buffers are needed (the finishers have cleared the
+            // scratch): the first thread makes sure of it on behalf of all, before the barrier.
+            if (tid == 0 && u >= 1) pipe_wait(ctrl, &ctrl->afree[b], static_cast<unsigned>(u - 1) & 1u);
             G.sync();
             amax = __uint_as_float(ctrl->amax[i % 3]);
             const float s = (amax < 0x1p-100f) ? 1.0f : __fdiv_rn(amax, static_cast<float>(qmax));
-            // only now are the set's other buffers needed: the finishers have cleared the scratch
-            if (u >= 1) pipe_wait_warp(ctrl, &ctrl->afree[b], static_cast<unsigned>(u - 1) & 1u);
             if (tid == 0) {
                 ctrl->scale[b] = s;
                 ctrl->fitem[b] = item;

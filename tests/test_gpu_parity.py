@@ -216,10 +216,21 @@ def test_more_layers_than_one_launch_table_holds():
         assert_layer_equal(b, w, 4, EKC, tag=f"layer {i} {shapes[i]}")
 
 
+def test_more_long_channel_layers_than_one_launch_table_holds():
+    """The same for the pipelined kernel: 101 layers of long 3x3 channels, two launches."""
+    shapes = [(1 + (i % 3), 912 + 4 * (i % 11), 3, 3) for i in range(101)]
+    ws = [W.random_layer(s, seed=3000 + i) for i, s in enumerate(shapes)]
+    n0 = sq.squant_launch_count()
+    bufs = run_gpu(ws, 4, EKC)
+    assert sq.squant_launch_count() == n0 + 2
+    for i, (b, w) in enumerate(zip(bufs, ws)):
+        assert_layer_equal(b, w, 4, EKC, tag=f"layer {i} {shapes[i]}")
+
+
 def test_non_finite_inputs_do_not_disturb_other_channels():
     """NaN / Inf weights are outside the method's domain; their channels produce unspecified
     codes, but every index the kernel forms stays in bounds and finite channels are unaffected."""
-    for shape in [(8, 64, 3, 3), (8, 256, 1, 1), (8, 10, 5, 5), (8, 2048, 3, 3)]:
+    for shape in [(8, 64, 3, 3), (8, 256, 1, 1), (8, 10, 5, 5), (8, 2048, 3, 3), (8, 1000, 3, 3), (300, 1024, 3, 3)]:
         w = W.random_layer(shape, seed=77)
         bad = w.copy()
         bad[1].reshape(-1)[3] = np.nan
