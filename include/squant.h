@@ -126,10 +126,13 @@ int squant_quantize_model(const squant_layer *layers, int32_t n_layers, const sq
                           void *cuda_stream);
 
 /*
- * The same, with HOST buffers: copies the weights to the current device, runs the grouped
- * launch, copies codes / scales / error sums back and waits for the stream.  Device staging
- * memory is cached inside the library between calls.  Pinned host memory gives the copies
- * their full speed; pageable memory works.
+ * The same, with HOST buffers: copies the weights to the current device, runs the launches,
+ * copies codes / scales / error sums back and returns when the outputs are in host memory.
+ * The layers are taken in chunks of about 64 MB of weights: uploads, launches and downloads of
+ * consecutive chunks overlap on two copy streams of the library (created on first use) beside
+ * the caller's stream, on which the launches run.  Device staging memory is cached inside the
+ * library between calls (cudaMalloc on first use or growth; squant_shutdown frees it).  Pinned
+ * host memory gives the copies their full speed and lets them overlap; pageable memory works.
  */
 int squant_quantize_model_host(const squant_layer *layers, int32_t n_layers,
                                const squant_options *opt, void *cuda_stream);

@@ -356,6 +356,36 @@ int launch_plan(const ParamPlan &p, cudaStream_t stream)
 struct Arena { void *ptr = nullptr; size_t bytes = 0; };
 std::vector<Arena> g_arenas;
 
+// Copy streams and events of the host-buffer entry point, one set per device, created on first
+// use: uploads, kernels and downloads of consecutive chunks of layers overlap.
+struct HostPipe {
+    cudaStream_t in = nullptr, out = nullptr;
+    cudaEvent_t start = nullptr;
+    std::vector<cudaEvent_t> uploaded, computed;
+};
+std::vector<HostPipe> g_host_pipes;
+constexpr size_t kHostChunkBytes = 64u << 20;   // weights per chunk: large enough to hide the launches
+
+int host_pipe(int device, size_t chunks, HostPipe *&out)
+{
+    if (static_cast<int>(g_host_pipes.size()) <= device) g_host_pipes.resize(device + 1);
+    HostPipe &hp = g_host_pipes[device];
+    if (!hp.in) {
+        SQ_CUDA(cudaStreamCreateWithFlags(&hp.in, cudaStreamNonBlocking));
+        SQ_CUDA(cudaStreamCreateWithFlags(&hp.out, cudaStreamNonBlocking));
+        SQ_CUDA(cudaEventCreateWithFlags(&hp.start, cudaEventDisableTiming));
+    }
+    while (hp.uploaded.size() < chunks) {
+        cudaEvent_t a = nullptr, b = nullptr;
+        SQ_CUDA(cudaEventCreateWithFlags(&a, cudaEventDisableTiming));
+        SQ_CUDA(cudaEventCreateWithFlags(&b, cudaEventDisableTiming));
+        hp.uploaded.push_back(a);
+        hp.computed.push_back(b);
+    }
+    out = &hp;
+    return SQUANT_OK;
+}
+
 inline size_t align256(size_t v) { return (v + 255) & ~static_cast<size_t>(255); }
 
 // ---- launch table of squant_quantize_layer_noalloc: part of the library image, never allocated.
@@ -442,34 +472,66 @@ int squant_quantize_model_host(const squant_layer *layers, int32_t n_layers,
     unsigned char *base = static_cast<unsigned char *>(a.ptr);
     for (int i = 0; i < n_layers; ++i) {
         const squant_layer &l = layers[i];
-        const size_t n = static_cast<size_t>(l.cin) * l.kh * l.kw * l.cout;
         dev[i].w = reinterpret_cast<const float *>(base + off[6 * i + 0]);
         dev[i].codes = reinterpret_cast<int8_t *>(base + off[6 * i + 1]);
         dev[i].scales = reinterpret_cast<float *>(base + off[6 * i + 2]);
         dev[i].kernel_err = l.kernel_err ? reinterpret_cast<float *>(base + off[6 * i + 3]) : nullptr;
         dev[i].channel_err = l.channel_err ? reinterpret_cast<float *>(base + off[6 * i + 4]) : nullptr;
         dev[i].dequant = l.dequant ? reinterpret_cast<float *>(base + off[6 * i + 5]) : nullptr;
-        SQ_CUDA(cudaMemcpyAsync(base + off[6 * i + 0], l.w, n * 4, cudaMemcpyHostToDevice, stream));
     }
-    const ParamPlan *pp = nullptr;
-    rc = get_plan(dev.data(), n_layers, o, pp);
-    if (rc) return rc;
-    rc = launch_plan(*pp, stream);
-    if (rc) return rc;
-    for (int i = 0; i < n_layers; ++i) {
-        const squant_layer &l = layers[i];
-        const size_t n = static_cast<size_t>(l.cin) * l.kh * l.kw * l.cout;
-        const size_t code_bytes = (o.flags & SQUANT_FLAG_PACK_INT4)
-                                      ? static_cast<size_t>(l.cout) * ((static_cast<size_t>(l.cin) * l.kh * l.kw + 1) / 2) : n;
-        SQ_CUDA(cudaMemcpyAsync(l.codes, dev[i].codes, code_bytes, cudaMemcpyDeviceToHost, stream));
-        SQ_CUDA(cudaMemcpyAsync(l.scales, dev[i].scales, static_cast<size_t>(l.cout) * 4, cudaMemcpyDeviceToHost, stream));
-        if (l.kernel_err)
-            SQ_CUDA(cudaMemcpyAsync(l.kernel_err, dev[i].kernel_err, static_cast<size_t>(l.cout) * l.cin * 4, cudaMemcpyDeviceToHost, stream));
-        if (l.channel_err)
-            SQ_CUDA(cudaMemcpyAsync(l.channel_err, dev[i].channel_err, static_cast<size_t>(l.cout) * 4, cudaMemcpyDeviceToHost, stream));
-        if (l.dequant)
-            SQ_CUDA(cudaMemcpyAsync(l.dequant, dev[i].dequant, n * 4, cudaMemcpyDeviceToHost, stream));
+    // Chunks of consecutive layers (about kHostChunkBytes of weights each).  Uploads run on one
+    // copy stream, each chunk's launches on the caller's stream once its upload is done, its
+    // downloads on a second copy stream once its launches are done: the two copy directions and
+    // the kernels overlap.
+    std::vector<int> chunk_first(1, 0);
+    {
+        size_t acc = 0;
+        for (int i = 0; i < n_layers; ++i) {
+            acc += static_cast<size_t>(layers[i].cin) * layers[i].kh * layers[i].kw * layers[i].cout * 4;
+            if (acc >= kHostChunkBytes && i + 1 < n_layers) { chunk_first.push_back(i + 1); acc = 0; }
+        }
+        chunk_first.push_back(n_layers);
     }
+    const size_t chunks = chunk_first.size() - 1;
+    HostPipe *hp = nullptr;
+    rc = host_pipe(device, chunks, hp);
+    if (rc) return rc;
+    SQ_CUDA(cudaEventRecord(hp->start, stream));          // uploads follow what the caller's stream holds so far
+    SQ_CUDA(cudaStreamWaitEvent(hp->in, hp->start, 0));
+    for (size_t c = 0; c < chunks; ++c) {
+        for (int i = chunk_first[c]; i < chunk_first[c + 1]; ++i) {
+            const squant_layer &l = layers[i];
+            const size_t n = static_cast<size_t>(l.cin) * l.kh * l.kw * l.cout;
+            SQ_CUDA(cudaMemcpyAsync(base + off[6 * i + 0], l.w, n * 4, cudaMemcpyHostToDevice, hp->in));
+        }
+        SQ_CUDA(cudaEventRecord(hp->uploaded[c], hp->in));
+    }
+    for (size_t c = 0; c < chunks; ++c) {
+        const int first = chunk_first[c], count = chunk_first[c + 1] - first;
+        SQ_CUDA(cudaStreamWaitEvent(stream, hp->uploaded[c], 0));
+        const ParamPlan *pp = nullptr;
+        rc = get_plan(dev.data() + first, count, o, pp);
+        if (rc) return rc;
+        rc = launch_plan(*pp, stream);
+        if (rc) return rc;
+        SQ_CUDA(cudaEventRecord(hp->computed[c], stream));
+        SQ_CUDA(cudaStreamWaitEvent(hp->out, hp->computed[c], 0));
+        for (int i = first; i < first + count; ++i) {
+            const squant_layer &l = layers[i];
+            const size_t n = static_cast<size_t>(l.cin) * l.kh * l.kw * l.cout;
+            const size_t code_bytes = (o.flags & SQUANT_FLAG_PACK_INT4)
+                                          ? static_cast<size_t>(l.cout) * ((static_cast<size_t>(l.cin) * l.kh * l.kw + 1) / 2) : n;
+            SQ_CUDA(cudaMemcpyAsync(l.codes, dev[i].codes, code_bytes, cudaMemcpyDeviceToHost, hp->out));
+            SQ_CUDA(cudaMemcpyAsync(l.scales, dev[i].scales, static_cast<size_t>(l.cout) * 4, cudaMemcpyDeviceToHost, hp->out));
+            if (l.kernel_err)
+                SQ_CUDA(cudaMemcpyAsync(l.kernel_err, dev[i].kernel_err, static_cast<size_t>(l.cout) * l.cin * 4, cudaMemcpyDeviceToHost, hp->out));
+            if (l.channel_err)
+                SQ_CUDA(cudaMemcpyAsync(l.channel_err, dev[i].channel_err, static_cast<size_t>(l.cout) * 4, cudaMemcpyDeviceToHost, hp->out));
+            if (l.dequant)
+                SQ_CUDA(cudaMemcpyAsync(l.dequant, dev[i].dequant, n * 4, cudaMemcpyDeviceToHost, hp->out));
+        }
+    }
+    SQ_CUDA(cudaStreamSynchronize(hp->out));
     SQ_CUDA(cudaStreamSynchronize(stream));
     return SQUANT_OK;
 }
@@ -599,6 +661,17 @@ int squant_shutdown(void)
         if (g_arenas[d].ptr) { cudaSetDevice(static_cast<int>(d)); cudaDeviceSynchronize(); cudaFree(g_arenas[d].ptr); }
     }
     g_arenas.clear();
+    for (size_t d = 0; d < g_host_pipes.size(); ++d) {
+        HostPipe &hp = g_host_pipes[d];
+        if (!hp.in) continue;
+        cudaSetDevice(static_cast<int>(d));
+        for (cudaEvent_t e : hp.uploaded) cudaEventDestroy(e);
+        for (cudaEvent_t e : hp.computed) cudaEventDestroy(e);
+        cudaEventDestroy(hp.start);
+        cudaStreamDestroy(hp.in);
+        cudaStreamDestroy(hp.out);
+    }
+    g_host_pipes.clear();
     if (have) cudaSetDevice(cur);
     return SQUANT_OK;
 }
