@@ -132,6 +132,36 @@ def test_long_3x3_channels_pipelined_kernel(bits, mode):
         assert_layer_equal(b, w, bits, mode, tag=f"second run shape{shapes[i]}")
 
 
+def test_random_mixed_launches():
+    """Seeded random models mixing long 3x3 layers (pipelined kernel), short 3x3, 1x1 and odd kernel
+    shapes, random bit widths and modes, each launched twice into the same buffers."""
+    rng = np.random.default_rng(12345)
+    for trial in range(12):
+        shapes = []
+        for _ in range(int(rng.integers(1, 7))):
+            kind = rng.integers(0, 4)
+            if kind == 0:
+                shapes.append((int(rng.integers(1, 400)), int(rng.integers(228, 513)) * 4, 3, 3))
+            elif kind == 1:
+                shapes.append((int(rng.integers(1, 40)), int(rng.integers(1, 228)) * 4, 3, 3))
+            elif kind == 2:
+                shapes.append((int(rng.integers(1, 60)), int(rng.integers(1, 3000)), 1, 1))
+            else:
+                shapes.append((int(rng.integers(1, 20)), int(rng.integers(1, 300)), int(rng.integers(1, 6)), int(rng.integers(1, 6))))
+        bits = int(rng.choice([2, 3, 4, 6, 8]))
+        mode = int(rng.choice([EKC, EK, EKC, EKC]))
+        ws = [adversarial_layer(s, seed=7000 + 10 * trial + i) for i, s in enumerate(shapes)]
+        bufs = run_gpu(ws, bits, mode)
+        for rep in range(2):
+            if rep:
+                for b in bufs:
+                    b.codes.fill_(-128)
+                sq.squant_quantize_model(bufs, bits=bits, mode=mode)
+                sq.squant_device_status()
+            for i, (b, w) in enumerate(zip(bufs, ws)):
+                assert_layer_equal(b, w, bits, mode, tag=f"trial {trial} run {rep} shape{shapes[i]} bits{bits} mode{mode}")
+
+
 @pytest.mark.parametrize("name,bits", [("resnet18", 4), ("resnet50", 4), ("resnet50", 6), ("mobilenetv2", 4),
                                        ("mixed_kernels", 4)])
 def test_model_configs_full(name, bits):
