@@ -621,7 +621,20 @@ __device__ __forceinline__ float stage_channel(const LayerDesc &L, int m, const 
             *reinterpret_cast<unsigned *>(red + 216) = 0u;               // absmax slot
         }
     }
-    if ((reinterpret_cast<uintptr_t>(wg) & 15) == 0 && (NK & 3) == 0) {
+    if (G.g == 32 && (reinterpret_cast<uintptr_t>(wg) & 15) == 0 && (NK & 3) == 0) {
+        // A channel of at most 1024 weights (one warp): plain 128-bit loads, all issued at once,
+        // arrive sooner than a bulk copy that is waited for through an mbarrier.
+        const int nv = NK >> 2;
+        const float4 *src = reinterpret_cast<const float4 *>(wg);
+#pragma unroll 8
+        for (int i = G.t; i < nv; i += 32) {
+            const float4 t = __ldcs(src + i);
+            reinterpret_cast<float4 *>(wbuf)[i] = t;
+            amax = fmaxf(fmaxf(amax, fabsf(t.x)), fmaxf(fabsf(t.y), fmaxf(fabsf(t.z), fabsf(t.w))));
+        }
+        G.sync();   // staged weights and the zeroed scratch are visible
+        amax = group_absmax(G, amax, red);
+    } else if ((reinterpret_cast<uintptr_t>(wg) & 15) == 0 && (NK & 3) == 0) {
         if (G.t == 0) {   // one thread waits for the copy; the others wait for it at the barrier
             mbar_init(bar, 1);
             bulk_load(wbuf, wg, static_cast<unsigned>(NK) * 4u, bar);
@@ -724,7 +737,8 @@ __device__ __forceinline__ void emit_channel(const LayerDesc &L, int m, const Gr
     }
     unsigned char *cg = reinterpret_cast<unsigned char *>(L.codes) + static_cast<size_t>(m) * row;
     const bool aligned = (reinterpret_cast<uintptr_t>(cg) & 15) == 0;
-    if (aligned && (row & 15) == 0) {
+    const bool bulk = aligned && (row & 15) == 0 && G.g > 32;   // a one-warp group stores its few bytes itself
+    if (bulk) {
         if (G.t == 0) bulk_store(cg, src, static_cast<unsigned>(row));
     } else if (aligned) {
         const int nv = row >> 4;
@@ -736,7 +750,7 @@ __device__ __forceinline__ void emit_channel(const LayerDesc &L, int m, const Gr
     if (G.t == 0) {
         L.scales[m] = s;
         if (L.cerr) L.cerr[m] = __fmul_rn(__ll2float_rn(ec), 0x1p-30f);
-        bulk_store_wait();   // shared memory must stay intact until the bulk copy has read it
+        if (bulk) bulk_store_wait();   // shared memory must stay intact until the bulk copy has read it
     }
 }
 
