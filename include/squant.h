@@ -138,7 +138,7 @@ int squant_quantize_model_host(const squant_layer *layers, int32_t n_layers,
                                const squant_options *opt, void *cuda_stream);
 
 /*
- * Geometry of the grouped launch (one thread block per 512/g output channels) that covers
+ * Geometry of the grouped launch (one thread block per 256/g output channels) that covers
  * these descriptors, as squant_quantize_layer_noalloc issues it (pointers are not dereferenced
  * and may be NULL here).  squant_quantize_model itself sends layers of long 3x3 channels to its
  * pipelined kernel instead, whose grid is one block per multiprocessor.  Any output may be NULL.
@@ -163,7 +163,7 @@ int squant_plan_info(const squant_layer *layers, int32_t n_layers, const squant_
  *   layer, opt, cuda_stream   as for squant_quantize_layer; DEVICE pointers, caller-owned
  *
  * Limits: one layer per call, and the layer's launch must need at most SQUANT_NOALLOC_MAX_CTAS
- * thread blocks (one block handles 512/g output channels, g = 32..512 threads per channel by
+ * thread blocks (one block handles 256/g output channels, g = 32..256 threads per channel by
  * channel length; squant_plan_info reports the count).  A larger layer is rejected with
  * SQUANT_ERR_LIMIT before anything is launched; split it by output-channel range and call once
  * per part.

@@ -57,8 +57,7 @@ int group_size(int64_t nk)
     if (nk <= 1024) return 32;
     if (nk <= 2048) return 64;
     if (nk <= 4096) return 128;
-    if (nk <= 8192) return 256;
-    return 512;
+    return 256;
 }
 
 int validate(const squant_layer *layers, int32_t n_layers, const squant_options *opt,
@@ -170,7 +169,7 @@ int g_next_slot = 0;   // next work-counter slot of the pipelined kernel; guarde
 // int8 codes, and two buffer sets fit the shared memory of one SM.
 bool pipe_eligible(const squant_layer &l, const LayerDesc &d, const squant_options &o, int max_smem)
 {
-    if (d.K != 9 || (d.N & 3) != 0 || d.NK <= 8192 || d.g != sq::kCtaThreads) return false;
+    if (d.K != 9 || (d.N & 3) != 0 || d.NK <= 8192) return false;
     if (!(o.mode & SQUANT_MODE_K) || (o.flags & SQUANT_FLAG_PACK_INT4) || l.dequant) return false;
     if ((reinterpret_cast<uintptr_t>(l.w) & 15) || (reinterpret_cast<uintptr_t>(l.codes) & 15)) return false;
     return 2 * d.slice_bytes + sq::kPipeCtrlBytes <= max_smem;

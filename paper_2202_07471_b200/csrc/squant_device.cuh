@@ -15,7 +15,7 @@
 
 namespace sq {
 
-constexpr int kCtaThreads = 512;
+constexpr int kCtaThreads = 256;   // four CTAs per SM (64 registers): measured best for whole models against 512 x 2 and 128 x 8
 constexpr int kOne = 1 << 30;   // perturbation 1.0 in fixed point
 constexpr int kHalf = 1 << 29;  // perturbation 0.5
 constexpr int kHistBins = 256;
@@ -31,13 +31,13 @@ struct LayerDesc {
     float *cerr;
     float *deq;
     int32_t M, N, K, NK;
-    int32_t g;            // threads per channel group: 32, 64, 128, 256 or 512
+    int32_t g;            // threads per channel group: 32, 64, 128 or 256
     int32_t g_shift;      // log2(g)
     int32_t slice_bytes;  // shared memory per group
     int32_t off_codes, off_ev, off_vv, off_vi, off_hist, off_red;
 };
 
-// One CTA: channels ch0 .. ch0 + 512/g - 1 of one layer, one per group.
+// One CTA: channels ch0 .. ch0 + 256/g - 1 of one layer, one per group.
 struct Item {
     int32_t layer;
     int32_t ch0;
@@ -46,7 +46,7 @@ struct Item {
 // Everything a grouped launch needs, passed BY VALUE as a kernel parameter: the descriptors sit
 // in the constant bank, so a CTA finds its work without a single global load (and nothing has
 // to be allocated or uploaded).  Work items of layer l are the CTAs first_item[l] ..
-// first_item[l+1]-1; item i of a layer handles channels i * (512 / g) ... of it.
+// first_item[l+1]-1; item i of a layer handles channels i * (256 / g) ... of it.
 constexpr int kMaxParamLayers = 96;
 struct LaunchTable {
     int n_layers;
@@ -1283,7 +1283,7 @@ __global__ void selfcheck_division_kernel(const float *scales, int n, int qmax,
 // One CTA per work item.  The descriptor of the CTA's layer comes either from the launch table
 // in the kernel's parameter space (kParams) or from a table in global memory.
 #ifndef SQ_MIN_CTAS
-#define SQ_MIN_CTAS 2
+#define SQ_MIN_CTAS 4
 #endif
 __device__ __forceinline__ void run_item(const LayerDesc &L, int ch0, unsigned char *smem, int qmax,
                                          unsigned mode)

@@ -36,13 +36,13 @@ def _info(shapes, **kw):
 def test_plan_geometry_for_the_five_configs():
     for name, wl in W.WORKLOADS.items():
         info = _info(wl.shapes)
-        assert info["cta_threads"] == 512
+        assert info["cta_threads"] == 256
         assert 0 < info["dynamic_smem_bytes"] <= 232448
         assert info["grid_ctas"] >= 1
     # one CTA per output channel for the large layers
     assert _info(W.WORKLOADS["large_layer"].shapes)["grid_ctas"] == 8 * 2048
     # small channels share a CTA: 16 warps, one channel each
-    assert _info([(64, 64, 3, 3)])["grid_ctas"] == 4
+    assert _info([(64, 64, 3, 3)])["grid_ctas"] == 8   # 64 channels, 8 one-warp groups per 256-thread block
     assert _info([(33, 1, 3, 3)])["grid_ctas"] == 3
 
 
