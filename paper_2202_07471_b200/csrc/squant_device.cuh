@@ -1193,7 +1193,7 @@ __device__ __forceinline__ void channel_body_k9_fast(const LayerDesc &L, int m, 
 // Fully connected and pointwise layers (K = 1; needs N % 4 = 0 and 2^-60 <= s <= 2^60).  Every
 // element is its own kernel, SQuant-K is a no-op (Sec. 3.4) and the element's perturbation is its
 // own candidate for SQuant-C.  A thread takes four elements at a time: one 128-bit shared load,
-// the reciprocal-based SQuant-E, one packed word of codes, and the four integer perturbations
+// the reciprocal-based SQuant-E (packed fp32x2), one packed word of codes, and the four integer perturbations
 // written back in place of the weights (they are the e' / v arrays of the channel step).
 __device__ __forceinline__ void channel_body_k1_fast(const LayerDesc &L, int m, const Group &G,
                                                      unsigned char *slice, float s, unsigned mode)
@@ -1207,16 +1207,16 @@ __device__ __forceinline__ void channel_body_k1_fast(const LayerDesc &L, int m, 
     const float s2 = __fmul_rn(s, 0x1p-30f);
     const float y = __frcp_rn(s2);
     const int quads = N >> 2;
+    const E2 c2 = make_e2(y, s2);
     long long esum = 0;
     for (int Q = G.t; Q < quads; Q += G.g) {
         const float4 w = wbuf4[Q];
-        unsigned t0, t1, t2, t3;
-        int4 P;
-        squant_e_fast(w.x, y, s2, t0, P.x);
-        squant_e_fast(w.y, y, s2, t1, P.y);
-        squant_e_fast(w.z, y, s2, t2, P.z);
-        squant_e_fast(w.w, y, s2, t3, P.w);
-        cbuf32[Q] = __byte_perm(__byte_perm(t0, t1, 0x0040), __byte_perm(t2, t3, 0x0040), 0x5410);
+        float2 ta, tb, Pa, Pb;
+        squant_e_fast2(make_float2(w.x, w.y), c2, ta, Pa);
+        squant_e_fast2(make_float2(w.z, w.w), c2, tb, Pb);
+        const int4 P = make_int4(__float2int_rn(Pa.x), __float2int_rn(Pa.y), __float2int_rn(Pb.x), __float2int_rn(Pb.y));
+        cbuf32[Q] = __byte_perm(__byte_perm(__float_as_uint(ta.x), __float_as_uint(ta.y), 0x0040),
+                                __byte_perm(__float_as_uint(tb.x), __float_as_uint(tb.y), 0x0040), 0x5410);
         reinterpret_cast<int4 *>(wbuf4)[Q] = P;
         if (mode & 4u) {
             hist_add(hist, P.x);
