@@ -1,6 +1,7 @@
 """Compile the CUDA library for sm_100a into paper_2202_07471_b200/libsquant.so (in-tree)."""
 from __future__ import annotations
 
+import glob
 import os
 import shutil
 import subprocess
@@ -10,7 +11,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsquant.so")
 SOURCES = [os.path.join(CSRC, "squant.cu")]
-DEPS = SOURCES + [os.path.join(CSRC, "squant_device.cuh"), os.path.join(ROOT, "include", "squant.h")]
+DEPS = SOURCES + sorted(glob.glob(os.path.join(CSRC, "*.cuh"))) + [os.path.join(ROOT, "include", "squant.h")]
 
 # -fmad=false: the solver's fp32 steps (division, rounding, difference) are written with
 # explicit round-to-nearest intrinsics; no contraction is wanted anywhere else either.

@@ -81,6 +81,7 @@ __device__ __forceinline__ void mbar_init(void *bar, unsigned count)
 {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the initialised barrier is visible to the async proxy
 }
 
 // One-dimensional bulk copy global -> shared of `bytes` (multiple of 16, both sides 16-byte
@@ -886,8 +887,9 @@ constexpr int kListCap = 128;   // the boundary list lives in the histogram's 1 
 
 __device__ __forceinline__ void hist_add(int *hist, int v)
 {
-    const int a = v < 0 ? -v : v;   // < 2^30 for every valid candidate; clamped for garbage input
-    atomicAdd(&hist[min(a >> 22, kHistBins - 1)], (v > 0 ? 1 : 0) | (v < 0 ? 0x10000 : 0));
+    // |v| < 2^30 for every valid candidate; unsigned arithmetic keeps the bin in range for garbage input too
+    const unsigned a = v < 0 ? 0u - static_cast<unsigned>(v) : static_cast<unsigned>(v);
+    atomicAdd(&hist[min(a >> 22, static_cast<unsigned>(kHistBins - 1))], (v > 0 ? 1 : 0) | (v < 0 ? 0x10000 : 0));
 }
 
 // Second half of a fast-path channel: channel sum, SQuant-C by the candidate histogram, flips,
@@ -1156,9 +1158,9 @@ __device__ __forceinline__ long long k9_quantize(const LayerDesc &L, int m, cons
                 const int pos = atomicAdd(redo_cnt, 1);
                 if (pos < redo_cap) redo[pos] = static_cast<unsigned short>(4 * Q + kq);
             }
-            {   // candidate histogram; |v| < 2^30, so the bin is in range (v = 0 adds nothing)
+            {   // candidate histogram; |v| < 2^30 for valid input, the mask keeps garbage in range (v = 0 adds nothing)
                 const int v = v4[kq];
-                atomicAdd(&hist[abs(v) >> 22], v > 0 ? 1 : ((v >> 31) & 0x10000));
+                atomicAdd(&hist[(abs(v) >> 22) & (kHistBins - 1)], v > 0 ? 1 : ((v >> 31) & 0x10000));
             }
             i4 |= idx << (8 * kq);
         }
