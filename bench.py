@@ -11,6 +11,10 @@ far larger than L2), 4 bit, E+K+C, one grouped kernel launch per step.
 With N > 1 (torchrun, one rank per GPU) every rank quantizes its own copy of the workload
 (different seed); there is no data-path collective, only the timing barrier and a MAX reduce.
 Prints ONE JSON line on rank 0.
+
+At N = 1 the outputs that were timed are then compared, channel by channel, with the CPU checker
+run over the whole workload on all host cores ("parity"), the checker is timed single-threaded on
+a sample ("cpu_baseline") and every other configuration is timed and checked in full ("configs").
 """
 from __future__ import annotations
 
@@ -51,6 +55,16 @@ def source_digest() -> str:
     return h.hexdigest()[:16]
 
 
+def nominal_peak_gbs() -> float:
+    """HBM peak as the profiler states it: DRAM bytes per second of the committed capture divided
+    by its own percent-of-peak figure (falls back to the 8 TB/s of the data sheet)."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "traffic.json")) as fh:
+            return float(json.load(fh)["ncu_dram_peak_gbs"])
+    except Exception:
+        return 8000.0
+
+
 def measured_peak():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -76,7 +90,7 @@ def ncu_traffic():
 class ClockSampler(threading.Thread):
     """Samples SM clock and throttle reasons through NVML while the timed region runs."""
 
-    def __init__(self, index: int, period_s: float = 0.005):
+    def __init__(self, index: int, period_s: float = 0.002):
         super().__init__(daemon=True)
         self.index, self.period = index, period_s
         self.samples, self.reasons, self.max_mhz = [], set(), None
@@ -132,26 +146,65 @@ def physical_gpu_index(local: int) -> int:
 
 
 # ----------------------------------------------------------------------------- CPU checker arm
-def oracle_rate(wl, seed, budget_s, threads=8):
-    """Times the checker, as it stands, single-threaded on whole output channels of the workload
-    until `budget_s` seconds of checker time are spent (at least one slab).  Returns
+def _same_words(a, b) -> bool:
+    return np.array_equal(np.ascontiguousarray(a).view(np.uint32), np.ascontiguousarray(b).view(np.uint32))
+
+
+def oracle_single_thread(host, budget_s):
+    """Times the checker, as it stands, on ONE thread over whole output channels of the workload
+    (slabs of 128 channels, layer after layer) until `budget_s` seconds are spent.  Returns
     (weights, seconds, description)."""
     import oracle
-    from paper_2202_07471_b200 import workloads as W
-    done_w, done_t, slabs = 0, 0.0, 0
-    slab = 128                                       # output channels per slab
-    m_total = wl.shapes[0][0]
-    for layer in range(len(wl.shapes)):
-        for c0 in range(0, m_total, slab):
-            w = W.layer_weights(wl, layer, seed, channels=slice(c0, c0 + slab), threads=threads)
+    done_w, done_t, slabs, slab = 0, 0.0, 0, 128
+    for w in host:
+        for c0 in range(0, w.shape[0], slab):
+            part = w[c0:c0 + slab]
             t0 = time.perf_counter()
-            oracle.quantize_layer(w, bits=BITS, mode=oracle.MODE_EKC)
+            oracle.quantize_layer(part, bits=BITS, mode=oracle.MODE_EKC)
             done_t += time.perf_counter() - t0
-            done_w += w.size
+            done_w += part.size
             slabs += 1
             if done_t >= budget_s:
-                return done_w, done_t, f"{slabs} slabs of {slab} output channels ({done_w} weights) of {wl.name}"
-    return done_w, done_t, f"all {done_w} weights of {wl.name}"
+                return done_w, done_t, f"{slabs} slabs of {slab} output channels ({done_w} weights), 1 thread"
+    return done_w, done_t, f"all {done_w} weights, 1 thread"
+
+
+def oracle_check_all(host, outs, bits, mode, threads, slab=64):
+    """Runs the checker over EVERY output channel of the given layers (numpy weights `host`) on
+    `threads` host threads - channels are independent sub-problems, so the split changes nothing -
+    and compares each slab with every output set in `outs` (lists of per-layer tuples
+    (codes, scales, kernel_err, channel_err) of numpy arrays).  Returns (channels, mismatching
+    channels per output set, seconds of wall clock)."""
+    import oracle
+    from concurrent.futures import ThreadPoolExecutor
+    jobs = [(i, c0) for i, w in enumerate(host) for c0 in range(0, w.shape[0], slab)]
+
+    def work(job):
+        i, c0 = job
+        r = oracle.quantize_layer(host[i][c0:c0 + slab], bits=bits, mode=mode)
+        bad = []
+        for o in outs:
+            codes, scales, kerr, cerr = o[i]
+            ok = (np.array_equal(codes[c0:c0 + slab], r.codes) and _same_words(scales[c0:c0 + slab], r.scales)
+                  and _same_words(kerr[c0:c0 + slab], r.kernel_err) and _same_words(cerr[c0:c0 + slab], r.channel_err))
+            if ok:
+                bad.append(0)
+            else:   # count the channels of the slab that differ anywhere
+                n = r.codes.shape[0]
+                d = np.zeros(n, dtype=bool)
+                d |= (codes[c0:c0 + slab].reshape(n, -1) != r.codes.reshape(n, -1)).any(1)
+                d |= scales[c0:c0 + slab].view(np.uint32) != r.scales.view(np.uint32)
+                d |= (kerr[c0:c0 + slab].view(np.uint32) != r.kernel_err.view(np.uint32)).any(1)
+                d |= cerr[c0:c0 + slab].view(np.uint32) != r.channel_err.view(np.uint32)
+                bad.append(int(d.sum()))
+        return bad
+
+    t0 = time.perf_counter()
+    with ThreadPoolExecutor(max_workers=threads) as ex:   # the checker is C code called through ctypes: the GIL is released
+        res = list(ex.map(work, jobs))
+    dt = time.perf_counter() - t0
+    channels = sum(w.shape[0] for w in host)
+    return channels, [sum(r[k] for r in res) for k in range(len(outs))], dt
 
 
 def run_reference(args):
@@ -185,6 +238,29 @@ def run_reference(args):
 
 
 # ----------------------------------------------------------------------------- CUDA arm
+def _to_host(bufs):
+    return [(b.codes.cpu().numpy(), b.scales.cpu().numpy(), b.kernel_err.cpu().numpy(), b.channel_err.cpu().numpy()) for b in bufs]
+
+
+def time_model(sq, torch, bufs, bits, mode, stream, flush, reps=15):
+    """One call over all layers: median milliseconds with L2 flushed before every call, and warm."""
+    call = sq.ModelCall(bufs, bits=bits, mode=mode)
+    for _ in range(3):
+        call.run(stream)
+    out = {}
+    for kind in ("cold", "warm"):
+        lat = []
+        for _ in range(reps):
+            if kind == "cold":
+                flush.fill_(1)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream); call.run(stream); b.record(stream)
+            torch.cuda.synchronize()
+            lat.append(a.elapsed_time(b))
+        out[kind] = statistics.median(lat)
+    return out
+
+
 def run_cuda(args):
     import torch
     import paper_2202_07471_b200 as sq
@@ -254,36 +330,59 @@ def run_cuda(args):
     e2e_s = D.max_over_ranks(time.perf_counter() - t0)
     h2d = sum(t.numel() * 4 for t in host)
     d2h = sum(b.codes.numel() + b.scales.numel() * 4 + b.kernel_err.numel() * 4 + b.channel_err.numel() * 4 for b in hb)
-    same = all(torch.equal(a.codes.cpu(), b.codes) for a, b in zip(dev[:1], hb[:1]))
 
-    # ---- latency of a whole small model in one launch (ResNet-50-shaped, L2 flushed before each)
     extra = {}
     if world == 1:
-        r50 = W.WORKLOADS["resnet50"]
-        rb = [sq.alloc_outputs(torch.from_numpy(W.layer_weights(r50, i, 0, threads=ncpu)).cuda()) for i in range(len(r50.shapes))]
-        rcall = sq.ModelCall(rb, bits=BITS, mode=sq.MODE_EKC)
+        # ---- the other configurations: whole model in one call, L2 cold and warm, every element
+        # compared with the checker; and the E|C ablation on one large layer (its channel step
+        # selects among all N*K elements)
         flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
-        for _ in range(3):
-            rcall.run(stream)
-        lat = []
-        for _ in range(20):
-            flush.fill_(1)
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(stream); rcall.run(stream); b.record(stream)
-            torch.cuda.synchronize()
-            lat.append(a.elapsed_time(b))
-        extra = {"resnet50_model_latency_ms": {"median": statistics.median(lat), "min": min(lat),
-                                               "weights": r50.n_weights, "layers": len(r50.shapes),
+        peak, _ = measured_peak()
+        cfgs = {}
+        for name, bits in (("single_conv", 4), ("resnet18", 4), ("resnet50", 4), ("resnet50", 6), ("mobilenetv2", 4),
+                           ("mixed_kernels", 4)):
+            w2 = W.WORKLOADS[name]
+            hw = [W.layer_weights(w2, i, 0, threads=ncpu) for i in range(len(w2.shapes))]
+            bufs = [sq.alloc_outputs(torch.from_numpy(x).cuda()) for x in hw]
+            t = time_model(sq, torch, bufs, bits, sq.MODE_EKC, stream, flush)
+            ch, bad, _ = oracle_check_all(hw, [_to_host(bufs)], bits, sq.MODE_EKC, ncpu)
+            alg = algorithmic_bytes(w2.shapes)
+            cfgs[name + ("" if bits == 4 else f"_{bits}bit")] = {
+                "layers": len(w2.shapes), "weights": w2.n_weights, "bits": bits, "ms_cold": t["cold"], "ms_warm": t["warm"],
+                "weights_per_s_cold": w2.n_weights / (t["cold"] * 1e-3), "gbs_cold": alg / (t["cold"] * 1e-3) / 1e9,
+                "frac_of_measured_cold": alg / (t["cold"] * 1e-3) / 1e9 / peak, "channels": ch, "mismatches": bad[0]}
+            del bufs
+        one = torch.from_numpy(host[0].numpy()).cuda()
+        eb = [sq.alloc_outputs(one)]
+        mode_ec = sq.MODE_E | sq.MODE_C
+        t = time_model(sq, torch, eb, BITS, mode_ec, stream, flush, reps=7)
+        ch, bad, _ = oracle_check_all([host[0].numpy()[:256]], [[tuple(a[:256] for a in _to_host(eb)[0])]], BITS, mode_ec, ncpu)
+        cfgs["large_layer_one_layer_E|C"] = {"layers": 1, "weights": one.numel(), "bits": BITS, "ms_cold": t["cold"], "ms_warm": t["warm"],
+                                             "weights_per_s_cold": one.numel() / (t["cold"] * 1e-3), "channels": ch, "mismatches": bad[0],
+                                             "note": "checker compared on the first 256 output channels"}
+        del eb, one, flush
+        r50 = cfgs["resnet50"]
+        extra = {"configs": cfgs,
+                 "resnet50_model_latency_ms": {"median": r50["ms_cold"], "weights": r50["weights"], "layers": r50["layers"],
                                                "l2": "flushed before each launch"}}
-        del rb, flush
 
     if rank != 0:
         D.finish()
         return
 
     peak, peak_kind = measured_peak()
+    nominal = nominal_peak_gbs()
     alg = algorithmic_bytes(wl.shapes)
     achieved = alg / (kernel_ms * 1e-3) / 1e9
+    traffic = ncu_traffic()
+    roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+            "frac": achieved / peak, "traffic": traffic, "peak_kind": f"of {peak_kind}",
+            "peak_ncu": nominal, "frac_of_ncu_peak": achieved / nominal,
+            "kernel": "squant_pipe_kernel", "kernel_ms": kernel_ms, "algorithmic_bytes_per_launch": alg}
+    if traffic:   # what actually crossed the DRAM interface (part of the output is still in L2 at kernel end)
+        roof["achieved_dram"] = traffic / (kernel_ms * 1e-3) / 1e9
+        roof["frac_dram_of_measured"] = roof["achieved_dram"] / peak
+        roof["frac_dram_of_ncu_peak"] = roof["achieved_dram"] / nominal
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps,
         "warmup": warmup, "ms_per_step": total_ms / steps, "higher_is_better": True,
@@ -293,18 +392,26 @@ def run_cuda(args):
                    "l2": "inputs (1.2 GB per step) larger than L2", "launches_per_step": 1},
         "clocks": clocks,
         "e2e": {"value": n_weights * world * e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
-                "d2h_bytes_per_step": d2h, "steps": e2e_steps, "matches_device_path": bool(same)},
+                "d2h_bytes_per_step": d2h, "steps": e2e_steps},
         "gpu_launches": int(launches),
-        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                     "frac": achieved / peak, "traffic": ncu_traffic(), "peak_kind": f"of {peak_kind}",
-                     "kernel": "squant_pipe_kernel", "kernel_ms": kernel_ms,
-                     "algorithmic_bytes_per_launch": alg},
+        "roofline": roof,
     }
     out.update(extra)
     if world == 1 and not args.no_cpu_baseline:
-        w_done, t_done, sample = oracle_rate(wl, 0, budget_s=args.cpu_budget, threads=ncpu)
+        # ---- the checker: one thread on a sample (the reported baseline), then all host cores over
+        # EVERY output channel, compared with the outputs of the timed device-resident run and of
+        # the host-buffer run
+        hnp = [t.numpy() for t in host]
+        w_done, t_done, sample = oracle_single_thread(hnp, budget_s=args.cpu_budget)
         out["cpu_baseline"] = {"value": w_done / t_done, "unit": UNIT, "cores": 1, "kind": "oracle",
-                               "sample": sample + ", 1 thread"}
+                               "sample": sample + f" of {wl.name}"}
+        dev_out = _to_host(dev)
+        hb_out = [(b.codes.numpy(), b.scales.numpy(), b.kernel_err.numpy(), b.channel_err.numpy()) for b in hb]
+        ch, bad, dt = oracle_check_all(hnp, [dev_out, hb_out], BITS, sq.MODE_EKC, ncpu)
+        out["cpu_baseline"]["all_cores"] = {"value": n_weights / dt, "unit": UNIT, "cores": ncpu,
+                                            "sample": f"all {n_weights} weights of {wl.name}, {ncpu} threads over slabs of output channels"}
+        out["parity"] = {"channels": ch, "mismatches": bad[0], "e2e_mismatches": bad[1],
+                         "what": "codes, scales, kernel_err, channel_err of every output channel of the timed runs against the CPU checker"}
     print(json.dumps(out))
     D.finish()
 
@@ -315,7 +422,7 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
-    ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of checker time for cpu_baseline")
+    ap.add_argument("--cpu-budget", type=float, default=8.0, help="seconds of single-thread checker time for cpu_baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -35,3 +35,25 @@ def test_algorithmic_bytes_of_the_bench_workload():
     wl = W.WORKLOADS[bench.WORKLOAD]
     # 3x3 layers: 4 B read + 1 B code + 4/9 B kernel sum per weight + 8 B per channel
     assert bench.algorithmic_bytes(wl.shapes) == 8 * (2048 * 2048 * 9 * 5 + 2048 * 2048 * 4 + 2048 * 8)
+
+
+def test_parity_checker_of_the_bench_counts_corrupted_channels():
+    """bench.py compares the timed outputs with the checker slab by slab on several threads; a
+    corrupted code, scale or error sum must be counted once per channel, clean outputs not at all."""
+    sys.path.insert(0, ROOT)
+    import numpy as np
+    import bench
+    import oracle
+    from paper_2202_07471_b200 import workloads as W
+    ws = [W.random_layer((70, 12, 3, 3), seed=1), W.random_layer((9, 40, 1, 1), seed=2)]
+    good = []
+    for w in ws:
+        r = oracle.quantize_layer(w, bits=4)
+        good.append((r.codes.copy(), r.scales.copy(), r.kernel_err.copy(), r.channel_err.copy()))
+    bad = [tuple(a.copy() for a in o) for o in good]
+    bad[0][0][3, 2, 1, 1] += 1          # one code of channel 3
+    bad[0][2][65, 7] = 0.25             # one kernel sum of channel 65 (second slab)
+    bad[1][1][8] *= 2.0                 # one scale
+    bad[1][3][8] = 0.125                # and the channel sum of the same channel: still one channel
+    ch, mism, dt = bench.oracle_check_all(ws, [good, bad], 4, oracle.MODE_EKC, threads=3, slab=64)
+    assert ch == 79 and mism == [0, 3] and dt > 0

@@ -324,3 +324,67 @@ def test_dequantized_output():
             r = oracle.quantize_layer(w, bits=4, mode=EKC, flags=flags, details=True)
             assert np.array_equal(b.dequant.cpu().numpy().view(np.uint32), r.dequant.view(np.uint32)), f"shape {shp}"
             assert np.array_equal(b.codes.cpu().numpy(), r.codes)
+
+
+def test_host_entry_point_several_chunks_against_the_checker():
+    """squant_quantize_model_host takes the layers in chunks of about 64 MB of weights whose
+    uploads, launches and downloads overlap on three streams.  Four layers of 75 MB (pipelined
+    kernel), a small one and a 1x1 one give five chunks; every output is compared with the checker
+    on a sample of whole channels of every layer, called twice (cached staging and plans)."""
+    shapes = [(512, 2048, 3, 3)] * 4 + [(40, 64, 3, 3), (300, 1000, 1, 1)]
+    ws = [W.random_layer(s, seed=900 + i) for i, s in enumerate(shapes)]
+    hb = [sq.alloc_outputs(torch.from_numpy(w).pin_memory(), pin=True) for w in ws]
+    for rep in range(2):
+        for b in hb:
+            b.codes.fill_(-128); b.scales.fill_(float("nan")); b.kernel_err.fill_(float("nan")); b.channel_err.fill_(float("nan"))
+        sq.squant_quantize_model_host(hb, bits=4)
+        sq.squant_device_status()
+        for i, (b, w) in enumerate(zip(hb, ws)):
+            pick = np.arange(0, w.shape[0], 7) if w.shape[0] > 100 else np.arange(w.shape[0])
+            r = oracle.quantize_layer(w[pick], bits=4)
+            assert np.array_equal(b.codes.numpy()[pick], r.codes), f"rep {rep} layer {i}"
+            assert np.array_equal(b.scales.numpy()[pick].view(np.uint32), r.scales.view(np.uint32))
+            assert np.array_equal(b.kernel_err.numpy()[pick].view(np.uint32), r.kernel_err.view(np.uint32))
+            assert np.array_equal(b.channel_err.numpy()[pick].view(np.uint32), r.channel_err.view(np.uint32))
+            assert int(b.codes.min()) >= -7 and not torch.isnan(b.scales).any()   # every channel was written
+
+
+@pytest.mark.parametrize("bits,flags", [(2, sq.FLAG_NARROW_RANGE), (6, sq.FLAG_NARROW_RANGE), (4, 0), (8, 0)])
+def test_pipelined_kernel_optional_outputs_and_ranges(bits, flags):
+    """Long 3x3 channels (pipelined kernel) without the optional outputs, at 2 and 6 bit, and
+    without the narrow-range flag; one table holds a layer with fewer channels than the GPU has
+    multiprocessors and one with many more."""
+    shapes = [(9, 1024, 3, 3), (700, 912, 3, 3), (33, 2048, 3, 3)]
+    ws = [adversarial_layer(s, seed=50 * bits + i) for i, s in enumerate(shapes)]
+    for variant in range(3):   # all outputs, no kernel sums, no sums at all
+        bufs = [sq.alloc_outputs(torch.from_numpy(w).cuda(), kernel_err=variant == 0, channel_err=variant <= 1) for w in ws]
+        for b in bufs:
+            b.codes.fill_(-128)
+        sq.squant_quantize_model(bufs, bits=bits, mode=EKC, flags=flags)
+        sq.squant_device_status()
+        for b, w, shp in zip(bufs, ws, shapes):
+            r = oracle.quantize_layer(w, bits=bits, mode=EKC, flags=flags)
+            assert np.array_equal(b.codes.cpu().numpy(), r.codes), f"{shp} variant {variant}"
+            assert np.array_equal(b.scales.cpu().numpy().view(np.uint32), r.scales.view(np.uint32))
+            if b.kernel_err is not None:
+                assert np.array_equal(b.kernel_err.cpu().numpy().view(np.uint32), r.kernel_err.view(np.uint32))
+            if b.channel_err is not None:
+                assert np.array_equal(b.channel_err.cpu().numpy().view(np.uint32), r.channel_err.view(np.uint32))
+
+
+def test_overlapping_calls_with_different_descriptors():
+    """Calls with different descriptors may overlap on the GPU: two models (both with layers for
+    the pipelined kernel, each with its own work counter) on two streams, several rounds."""
+    wa = [W.random_layer((200, 1024, 3, 3), seed=61), W.random_layer((50, 64, 3, 3), seed=62)]
+    wb = [W.random_layer((300, 912, 3, 3), seed=63), W.random_layer((64, 300, 1, 1), seed=64)]
+    ba = [sq.alloc_outputs(torch.from_numpy(w).cuda()) for w in wa]
+    bb = [sq.alloc_outputs(torch.from_numpy(w).cuda()) for w in wb]
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    for _ in range(5):
+        sq.squant_quantize_model(ba, bits=4, stream=s1)
+        sq.squant_quantize_model(bb, bits=4, stream=s2)
+    sq.squant_device_status()
+    for bufs, ws in ((ba, wa), (bb, wb)):
+        for b, w in zip(bufs, ws):
+            assert_layer_equal(b, w, 4, EKC)
