@@ -33,11 +33,11 @@ def _load():
     global _lib
     if _lib is None:
         lib = ctypes.CDLL(_build.build())
-        lib.sqo_quantize_layer.restype = ctypes.c_int
-        lib.sqo_quantize_layer.argtypes = [
+        lib.sqo_quantize_layer_scaled.restype = ctypes.c_int
+        lib.sqo_quantize_layer_scaled.argtypes = [
             ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
             ctypes.POINTER(_Options), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
-            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
         _lib = lib
     return _lib
 
@@ -54,8 +54,10 @@ class OracleResult:
 
 
 def quantize_layer(w: np.ndarray, bits: int = 4, mode: int = MODE_EKC,
-                   flags: int = FLAG_NARROW_RANGE, *, details: bool = False) -> OracleResult:
-    """Run the checker on one layer.  `w` is [M, N, kh, kw], [M, N, K] or [M, N] fp32."""
+                   flags: int = FLAG_NARROW_RANGE, *, details: bool = False,
+                   scales_in: Optional[np.ndarray] = None) -> OracleResult:
+    """Run the checker on one layer.  `w` is [M, N, kh, kw], [M, N, K] or [M, N] fp32.
+    scales_in ([M] fp32) replaces the absmax scales by the caller's (Algorithm 1's input s)."""
     w = np.ascontiguousarray(w, dtype=np.float32)
     if w.ndim < 2:
         raise ValueError("weights need at least [M, N]")
@@ -73,8 +75,13 @@ def quantize_layer(w: np.ndarray, bits: int = 4, mode: int = MODE_EKC,
     deq = np.empty(w.shape, dtype=np.float32) if details else None
     opt = _Options(bits, mode, flags)
     ptr = lambda a: a.ctypes.data_as(ctypes.c_void_p) if a is not None else None
-    rc = _load().sqo_quantize_layer(ptr(w), M, N, K, ctypes.byref(opt), ptr(codes), ptr(scales),
-                                    ptr(kerr), ptr(cerr), ptr(pert), ptr(flip), ptr(deq))
+    sin = None
+    if scales_in is not None:
+        sin = np.ascontiguousarray(scales_in, dtype=np.float32)
+        if sin.shape != (M,):
+            raise ValueError("scales_in needs one fp32 scale per output channel")
+    rc = _load().sqo_quantize_layer_scaled(ptr(w), M, N, K, ctypes.byref(opt), ptr(codes), ptr(scales),
+                                           ptr(kerr), ptr(cerr), ptr(pert), ptr(flip), ptr(deq), ptr(sin))
     if rc != 0:
         raise ValueError(f"sqo_quantize_layer failed with code {rc}")
     return OracleResult(codes, scales, kerr, cerr, pert, flip, deq)

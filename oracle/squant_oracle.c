@@ -19,6 +19,17 @@
  *          symmetric absmax, s_m = max|W[m]| / qmax in IEEE fp32, qmax = 2^(bits-1) - 1.
  *          A channel whose absmax is below 2^-100 (which includes the all-zero channel)
  *          gets s_m = 1, so every code is 0.
+ *          Algorithm 1 itself takes the scale vector as an INPUT, and Sec. 2.2 clips
+ *          round(w / s) to the integer range; with a caller-supplied scale (scales_in, one
+ *          per output channel) that clip really fires.  The paper says nothing about clipped
+ *          elements in SQuant-K / SQuant-C.  Reading used here: a clipped element keeps its
+ *          saturated code, its perturbation p = q - w/s (now possibly far beyond 0.5) enters
+ *          every kernel and channel sum like any other, and it can never be flipped outward
+ *          (the flipped code would leave the range), so it is never a candidate; when a
+ *          kernel or channel has fewer candidates than round(|e|) asks for, all of them are
+ *          flipped and the remaining |e| > 0.5 is what the error sums report.  A supplied
+ *          scale that is not a positive finite number is replaced by 1.  Perturbations are
+ *          held in 64 bits; |w / s| is assumed below 2^20.
  *
  *  E       Algorithm 1 "Scale and SQuant-E (Rounding)" / Eq. 9: x = w / s_m (IEEE fp32
  *          division), q = round-to-nearest(x) with ties to even, clipped to [qmin, qmax]
@@ -72,7 +83,7 @@ typedef struct {
 } sqo_options;
 
 typedef struct {
-    int32_t mag;  /* |perturbation| in units of 2^-30 */
+    int64_t mag;  /* |perturbation| in units of 2^-30 */
     int32_t idx;  /* flat index inside the output channel */
 } sqo_cand;
 
@@ -95,29 +106,36 @@ static int sqo_sign64(int64_t v) { return (v > 0) - (v < 0); }
 
 typedef struct {
     int32_t *q;      /* [N*K] integer codes */
-    int32_t *P;      /* [N*K] fixed-point perturbations */
+    int64_t *P;      /* [N*K] fixed-point perturbations */
     uint8_t *flip;   /* [N*K] bit0: flipped by SQuant-K, bit1: flipped by SQuant-C */
-    int32_t *cv;     /* [N*K] SQuant-C candidate value per slot (0 = none) */
+    int64_t *cv;     /* [N*K] SQuant-C candidate value per slot (0 = none) */
     int32_t *cj;     /* [N*K] SQuant-C candidate flat index per slot */
     sqo_cand *list;  /* [N*K] scratch for sorting */
 } sqo_work;
 
-static void sqo_channel(const float *w, int32_t N, int32_t K, const sqo_options *opt,
+static void sqo_channel(const float *w, int32_t N, int32_t K, const sqo_options *opt, const float *scale_in,
                         sqo_work *wk, int8_t *codes, float *scale_out,
                         float *kernel_err, float *channel_err, float *dequant)
 {
     const int32_t NK = N * K;
     const int32_t qmax = (1 << (opt->bits - 1)) - 1;
     const int32_t qmin = (opt->flags & SQO_FLAG_NARROW_RANGE) ? -qmax : -qmax - 1;
-    int32_t *q = wk->q, *P = wk->P;
+    int32_t *q = wk->q;
+    int64_t *P = wk->P;
 
-    /* scale: symmetric absmax */
-    float a = 0.0f;
-    for (int32_t j = 0; j < NK; ++j) {
-        float t = fabsf(w[j]);
-        if (t > a) a = t;
+    /* scale: the caller's (Algorithm 1 takes s as an input), else symmetric absmax */
+    float s;
+    if (scale_in) {
+        s = *scale_in;
+        if (!(s > 0.0f && s < INFINITY)) s = 1.0f;
+    } else {
+        float a = 0.0f;
+        for (int32_t j = 0; j < NK; ++j) {
+            float t = fabsf(w[j]);
+            if (t > a) a = t;
+        }
+        s = (a < 0x1p-100f) ? 1.0f : a / (float)qmax;
     }
-    const float s = (a < 0x1p-100f) ? 1.0f : a / (float)qmax;
     *scale_out = s;
 
     /* SQuant-E (Eq. 9): round to nearest, clip, perturbation, one conversion to fixed point */
@@ -128,7 +146,7 @@ static void sqo_channel(const float *w, int32_t N, int32_t K, const sqo_options 
         if (qf < (float)qmin) qf = (float)qmin;
         float p = qf - x;
         q[j] = (int32_t)qf;
-        P[j] = (int32_t)nearbyintf(p * 0x1p30f);
+        P[j] = (int64_t)nearbyint((double)p * 0x1p30);   /* exact: p is an fp32 number */
         wk->flip[j] = 0;
     }
 
@@ -136,7 +154,8 @@ static void sqo_channel(const float *w, int32_t N, int32_t K, const sqo_options 
     int32_t n_slots = 0;              /* number of SQuant-C candidate slots */
     if (opt->mode & SQO_MODE_K) {
         for (int32_t n = 0; n < N; ++n) {
-            int32_t *qk = q + (size_t)n * K, *Pk = P + (size_t)n * K;
+            int32_t *qk = q + (size_t)n * K;
+            int64_t *Pk = P + (size_t)n * K;
             int64_t e = 0;
             for (int32_t i = 0; i < K; ++i) e += Pk[i];
             wk->cv[n] = 0;
@@ -159,7 +178,7 @@ static void sqo_channel(const float *w, int32_t N, int32_t K, const sqo_options 
             for (int64_t r = 0; r < k; ++r) {
                 int32_t j = wk->list[r].idx;
                 q[j] -= sgn;
-                P[j] -= sgn * (int32_t)SQO_ONE;
+                P[j] -= sgn * SQO_ONE;
                 wk->flip[j] |= 1;
             }
             if (k * SQO_ONE > abs_e) {              /* Over SQuant: last flipped, post-flip value */
@@ -190,7 +209,8 @@ static void sqo_channel(const float *w, int32_t N, int32_t K, const sqo_options 
             const int64_t abs_e = ec > 0 ? ec : -ec;
             int32_t nc = 0;
             for (int32_t t = 0; t < n_slots; ++t) {
-                int32_t v = wk->cv[t], j = wk->cj[t];
+                int64_t v = wk->cv[t];
+                int32_t j = wk->cj[t];
                 int32_t flipped = q[j] - sgn;
                 if (sqo_sign64(v) == sgn && flipped >= qmin && flipped <= qmax) {
                     wk->list[nc].mag = v > 0 ? v : -v;
@@ -204,7 +224,7 @@ static void sqo_channel(const float *w, int32_t N, int32_t K, const sqo_options 
             for (int64_t r = 0; r < k; ++r) {
                 int32_t j = wk->list[r].idx;
                 q[j] -= sgn;
-                P[j] -= sgn * (int32_t)SQO_ONE;
+                P[j] -= sgn * SQO_ONE;
                 wk->flip[j] |= 2;
             }
         }
@@ -242,11 +262,13 @@ static void sqo_channel(const float *w, int32_t N, int32_t K, const sqo_options 
  *   pert         out [M][N][K] final fixed-point perturbations (2^-30 units), may be NULL
  *   flip         out [M][N][K] flip record (bit0 SQuant-K, bit1 SQuant-C), may be NULL
  *   dequant      out [M][N][K] fp32 code * scale (Algorithm 1's return value), may be NULL
- * Inputs must be finite.  Returns SQO_OK or a negative error.
+ *   scales_in    in  [M] caller-supplied scales (Algorithm 1's input s), may be NULL: absmax scales
+ * pert is the perturbation clamped to 32 bits (exact whenever no element is clipped by more than
+ * one step).  Inputs must be finite.  Returns SQO_OK or a negative error.
  */
-int sqo_quantize_layer(const float *w, int32_t M, int32_t N, int32_t K, const sqo_options *opt,
-                       int8_t *codes, float *scales, float *kernel_err, float *channel_err,
-                       int32_t *pert, uint8_t *flip, float *dequant)
+int sqo_quantize_layer_scaled(const float *w, int32_t M, int32_t N, int32_t K, const sqo_options *opt,
+                              int8_t *codes, float *scales, float *kernel_err, float *channel_err,
+                              int32_t *pert, uint8_t *flip, float *dequant, const float *scales_in)
 {
     if (!w || !opt || !codes || !scales || M < 0 || N <= 0 || K <= 0) return SQO_ERR_ARG;
     if (opt->bits < 2 || opt->bits > 8 || !(opt->mode & SQO_MODE_E)) return SQO_ERR_ARG;
@@ -255,9 +277,9 @@ int sqo_quantize_layer(const float *w, int32_t M, int32_t N, int32_t K, const sq
     const size_t NK = (size_t)N * K;
     sqo_work wk;
     wk.q = (int32_t *)malloc(NK * sizeof(int32_t));
-    wk.P = (int32_t *)malloc(NK * sizeof(int32_t));
+    wk.P = (int64_t *)malloc(NK * sizeof(int64_t));
     wk.flip = (uint8_t *)malloc(NK);
-    wk.cv = (int32_t *)malloc(NK * sizeof(int32_t));
+    wk.cv = (int64_t *)malloc(NK * sizeof(int64_t));
     wk.cj = (int32_t *)malloc(NK * sizeof(int32_t));
     wk.list = (sqo_cand *)malloc(NK * sizeof(sqo_cand));
     int rc = SQO_OK;
@@ -265,15 +287,27 @@ int sqo_quantize_layer(const float *w, int32_t M, int32_t N, int32_t K, const sq
         rc = SQO_ERR_NOMEM;
     } else {
         for (int32_t m = 0; m < M; ++m) {
-            sqo_channel(w + (size_t)m * NK, N, K, opt, &wk,
+            sqo_channel(w + (size_t)m * NK, N, K, opt, scales_in ? scales_in + m : NULL, &wk,
                         codes + (size_t)m * ((opt->flags & SQO_FLAG_PACK_INT4) ? (NK + 1) / 2 : NK), scales + m,
                         kernel_err ? kernel_err + (size_t)m * N : NULL,
                         channel_err ? channel_err + m : NULL,
                         dequant ? dequant + (size_t)m * NK : NULL);
-            if (pert) memcpy(pert + (size_t)m * NK, wk.P, NK * sizeof(int32_t));
+            if (pert)
+                for (size_t j = 0; j < NK; ++j) {
+                    int64_t v = wk.P[j];
+                    pert[(size_t)m * NK + j] = (int32_t)(v > INT32_MAX ? INT32_MAX : (v < INT32_MIN ? INT32_MIN : v));
+                }
             if (flip) memcpy(flip + (size_t)m * NK, wk.flip, NK);
         }
     }
     free(wk.q); free(wk.P); free(wk.flip); free(wk.cv); free(wk.cj); free(wk.list);
     return rc;
+}
+
+/* The same with absmax scales (no supplied scales). */
+int sqo_quantize_layer(const float *w, int32_t M, int32_t N, int32_t K, const sqo_options *opt,
+                       int8_t *codes, float *scales, float *kernel_err, float *channel_err,
+                       int32_t *pert, uint8_t *flip, float *dequant)
+{
+    return sqo_quantize_layer_scaled(w, M, N, K, opt, codes, scales, kernel_err, channel_err, pert, flip, dequant, NULL);
 }
