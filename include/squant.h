@@ -95,6 +95,17 @@ typedef struct squant_layer {
                                  perturbations */
     float *dequant;      /* out, may be NULL: [cout][cin][kh][kw] fp32 quantized weights
                                  code * s_m - what Algorithm 1 itself returns ("C * s") */
+    const float *scales_in; /* in, may be NULL: [cout] caller-supplied scales, the input s of
+                                 Algorithm 1.  NULL: absmax scales (above).  With a supplied scale
+                                 the clip of Sec. 2.2 really fires: a clipped element keeps its
+                                 saturated code, its perturbation enters the kernel and channel
+                                 sums, and it is never flipped outward; when fewer candidates exist
+                                 than round(|e|) asks for, all are flipped and kernel_err /
+                                 channel_err report what is left (then above 0.5).  A scale that
+                                 is not a positive finite number is replaced by 1; |w / s| must
+                                 stay below 2^12.  `scales` receives the scales used.  Not
+                                 available for E|C without K on kernels larger than 1x1
+                                 (SQUANT_ERR_MODE). */
 } squant_layer;
 
 /*

@@ -29,7 +29,7 @@
  *          kernel or channel has fewer candidates than round(|e|) asks for, all of them are
  *          flipped and the remaining |e| > 0.5 is what the error sums report.  A supplied
  *          scale that is not a positive finite number is replaced by 1.  Perturbations are
- *          held in 64 bits; |w / s| is assumed below 2^20.
+ *          held in 64 bits; |w / s| is assumed below 2^12.
  *
  *  E       Algorithm 1 "Scale and SQuant-E (Rounding)" / Eq. 9: x = w / s_m (IEEE fp32
  *          division), q = round-to-nearest(x) with ties to even, clipped to [qmin, qmax]

@@ -41,7 +41,7 @@ class Layer(ctypes.Structure):
     _fields_ = [("w", ctypes.c_void_p), ("cout", ctypes.c_int32), ("cin", ctypes.c_int32),
                 ("kh", ctypes.c_int32), ("kw", ctypes.c_int32), ("codes", ctypes.c_void_p),
                 ("scales", ctypes.c_void_p), ("kernel_err", ctypes.c_void_p),
-                ("channel_err", ctypes.c_void_p), ("dequant", ctypes.c_void_p)]
+                ("channel_err", ctypes.c_void_p), ("dequant", ctypes.c_void_p), ("scales_in", ctypes.c_void_p)]
 
 
 _lib = None
@@ -92,6 +92,7 @@ class LayerBuffers:
     kernel_err: Optional[torch.Tensor]
     channel_err: Optional[torch.Tensor]
     dequant: Optional[torch.Tensor] = None     # fp32 code * scale, shape of the weights
+    scales_in: Optional[torch.Tensor] = None   # fp32 [cout] caller-supplied scales (None: absmax scales)
 
 
 def alloc_outputs(w: torch.Tensor, kernel_err: bool = True, channel_err: bool = True,
@@ -124,7 +125,11 @@ def _descriptor(b: LayerBuffers) -> Layer:
     else:
         raise ValueError("weights must be [cout, cin], [cout, cin, k] or [cout, cin, kh, kw]")
     ptr = lambda t: t.data_ptr() if t is not None else None
-    return Layer(ptr(w), m, n, kh, kw, ptr(b.codes), ptr(b.scales), ptr(b.kernel_err), ptr(b.channel_err), ptr(b.dequant))
+    if b.scales_in is not None and (b.scales_in.dtype != torch.float32 or b.scales_in.numel() != m or not b.scales_in.is_contiguous()
+                                    or b.scales_in.device != w.device):
+        raise ValueError("scales_in must be a contiguous fp32 tensor [cout] next to the weights")
+    return Layer(ptr(w), m, n, kh, kw, ptr(b.codes), ptr(b.scales), ptr(b.kernel_err), ptr(b.channel_err), ptr(b.dequant),
+                 ptr(b.scales_in))
 
 
 def _options(bits: int, mode: int, flags: int) -> Options:
@@ -209,7 +214,7 @@ def squant_plan_info(shapes: Sequence[Sequence[int]], bits: int = 4, mode: int =
                      flags: int = FLAG_NARROW_RANGE) -> dict:
     """Launch geometry for layers of the given [cout, cin, kh, kw] shapes (no GPU needed)."""
     arr = (Layer * max(1, len(shapes)))(*[Layer(None, int(s[0]), int(s[1]), int(s[2]), int(s[3]),
-                                                None, None, None, None, None) for s in shapes])
+                                                None, None, None, None, None, None) for s in shapes])
     opt = _options(bits, mode, flags)
     g, t, s = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32()
     _check(load_library().squant_plan_info(arr, len(shapes), ctypes.byref(opt), ctypes.byref(g),

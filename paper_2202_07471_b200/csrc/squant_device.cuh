@@ -30,6 +30,7 @@ struct LayerDesc {
     float *kerr;
     float *cerr;
     float *deq;
+    const float *sin;     // caller-supplied scales, or null: absmax scales
     int32_t M, N, K, NK;
     int32_t g;            // threads per channel group: 32, 64, 128 or 256
     int32_t g_shift;      // log2(g)
@@ -688,7 +689,7 @@ __device__ __forceinline__ ChannelStep channel_step(const LayerDesc &L, const Gr
     if ((mode & 4u) && c.ec != 0) {
         c.sgn_c = c.ec > 0 ? 1 : -1;
         const long long abs_e = c.ec > 0 ? c.ec : -c.ec;
-        const int kc = flip_count(abs_e);
+        const int kc = static_cast<int>(min((abs_e + (kHalf - 1)) >> 30, 1ll << 30));   // a clipped channel's sum can be huge
         if (kc > 0) c.k_eff = select_threshold(G, vv, L.N, c.sgn_c, kc, hist, bc, c.T);
         c.ec -= static_cast<long long>(c.sgn_c) * c.k_eff * kOne;
     }
@@ -702,6 +703,7 @@ __device__ __forceinline__ ChannelStep channel_step(const LayerDesc &L, const Gr
 // low nibble = even flat index, ceil(N*K / 2) bytes per output channel, packed into `scratch`
 // (shared memory that is dead by now) first.  Aligned rows leave by one bulk asynchronous copy.
 constexpr unsigned kModePackInt4 = 0x100u;
+constexpr unsigned kModeWideRange = 0x200u;   // the clip range is [-qmax - 1, qmax] (no narrow-range flag)
 
 __device__ __forceinline__ void emit_channel(const LayerDesc &L, int m, const Group &G,
                                              const unsigned char *cbuf, unsigned char *scratch, float s,
@@ -823,6 +825,93 @@ __device__ __forceinline__ void channel_body(const LayerDesc &L, int m, const Gr
 
     // ---- codes, scale, channel error (the staged weights / perturbations are dead: scratch)
     emit_channel(L, m, G, reinterpret_cast<const unsigned char *>(cbuf), slice, s, ec, mode);
+}
+
+// ---------------------------------------------------------------- channel body, caller-supplied scale
+// With a supplied scale the clip of Sec. 2.2 fires, so nothing of what the other bodies assume
+// holds: a perturbation can be far beyond one half (it is summed in 64 bits; the 32-bit copy used
+// for the selection saturates, which is harmless because a clipped element is no candidate), an
+// element at the edge of the range cannot be flipped outward, and a kernel or channel can run
+// out of candidates before its sum is within one half.  Plain thread-per-kernel code, any kernel
+// size, IEEE division; correctness first.  The layer's slice keeps e', v and idx in arrays of
+// their own also for 1x1 kernels (the host lays such layers out that way).
+__device__ __forceinline__ void channel_body_clip(const LayerDesc &L, int m, const Group &G, unsigned char *slice, float s,
+                                                  unsigned mode, int qmax)
+{
+    const int K = L.K, N = L.N;
+    const int qmin = (mode & kModeWideRange) ? -qmax - 1 : -qmax;
+    float *wbuf = reinterpret_cast<float *>(slice);
+    int8_t *cbuf = reinterpret_cast<int8_t *>(slice + L.off_codes);
+    int *ev = reinterpret_cast<int *>(slice + L.off_ev);
+    int *vv = reinterpret_cast<int *>(slice + L.off_vv);
+    unsigned short *vi = reinterpret_cast<unsigned short *>(slice + L.off_vi);
+    const bool do_k = (mode & 2u) != 0;
+    float *kerr = L.kerr ? L.kerr + static_cast<size_t>(m) * N : nullptr;
+    long long esum = 0;
+    for (int n = G.t; n < N; n += G.g) {
+        float *wk = wbuf + static_cast<size_t>(n) * K;
+        int *Pk = reinterpret_cast<int *>(wk);   // the 32-bit perturbations overwrite the weights
+        int8_t *ck = cbuf + static_cast<size_t>(n) * K;
+        long long e = 0;
+        for (int i = 0; i < K; ++i) {
+            const float x = __fdiv_rn(wk[i], s);
+            const float qf = fminf(fmaxf(rintf(x), static_cast<float>(qmin)), static_cast<float>(qmax));   // the clip of Sec. 2.2
+            const long long P = __float2ll_rn(__fmul_rn(__fsub_rn(qf, x), 1073741824.0f));
+            ck[i] = static_cast<int8_t>(__float2int_rn(qf));
+            Pk[i] = static_cast<int>(max(min(P, 0x7fffffffll), -0x7fffffffll));
+            e += P;
+        }
+        int v = 0, idx = 0;
+        if (e != 0) {
+            const int sgn = e > 0 ? 1 : -1;
+            const long long abs_e = e > 0 ? e : -e;
+            const int k = do_k ? static_cast<int>(min((abs_e + (kHalf - 1)) >> 30, static_cast<long long>(K) + 1)) : 0;
+            int flips = 0, last = -1, cand = -1;
+            for (int r = 0; r <= k; ++r) {
+                int best = 0, bi = -1;
+                for (int i = 0; i < K; ++i) {
+                    const int key = sgn * Pk[i], fl = ck[i] - sgn;
+                    if (key > best && fl >= qmin && fl <= qmax) { best = key; bi = i; }
+                }
+                if (bi < 0) break;   // out of candidates: the kernel keeps what is left of its sum
+                if (r < k) {
+                    Pk[bi] -= sgn * kOne;
+                    ck[bi] = static_cast<int8_t>(ck[bi] - sgn);
+                    last = bi;
+                    ++flips;
+                } else {
+                    cand = bi;
+                }
+            }
+            e -= static_cast<long long>(sgn) * flips * kOne;
+            if (static_cast<long long>(flips) * kOne > abs_e) {   // Over SQuant: flip back candidate
+                idx = last;
+                v = Pk[last];
+            } else if (cand >= 0) {                               // Under SQuant: next un-flipped
+                idx = cand;
+                v = Pk[cand];
+            }
+        }
+        // a kernel that SQuant-C can flip has a candidate, hence |e'| <= 1/2: its 32-bit copy is exact
+        ev[n] = static_cast<int>(max(min(e, 0x7fffffffll), -0x7fffffffll));
+        vv[n] = v;
+        vi[n] = static_cast<unsigned short>(idx);
+        if (kerr) kerr[n] = __fmul_rn(__ll2float_rn(e), 0x1p-30f);
+        esum += e;
+    }
+    const ChannelStep cs = channel_step(L, G, slice, esum, mode);
+    if (cs.k_eff > 0) {
+        for (int n = G.t; n < N; n += G.g) {
+            const unsigned long long ck = cand_key(vv[n], cs.sgn_c, n);
+            if (ck != 0 && ck >= cs.T) {
+                const size_t j = static_cast<size_t>(n) * K + vi[n];
+                cbuf[j] = static_cast<int8_t>(cbuf[j] - cs.sgn_c);
+                if (kerr) kerr[n] = __fmul_rn(__int2float_rn(ev[n] - cs.sgn_c * kOne), 0x1p-30f);
+            }
+        }
+    }
+    G.sync();
+    emit_channel(L, m, G, reinterpret_cast<const unsigned char *>(cbuf), slice, s, cs.ec, mode);
 }
 
 // ---------------------------------------------------------------- channel body, E + C without K
@@ -1300,7 +1389,11 @@ __device__ __forceinline__ void run_item(const LayerDesc &L, int ch0, unsigned c
     unsigned char *slice = smem + static_cast<size_t>(gi) * L.slice_bytes;
     const float s = stage_channel(L, m, G, slice, qmax);
     if (s == 0.0f) return;   // staging wait ran out (status word set); nothing is written
-    if (L.K > 1 && (mode & 6u) == 4u) {   // E + C without K
+    if (L.sin) {   // Algorithm 1 with its scale as an input
+        float sc = L.sin[m];
+        if (!(sc > 0.0f && sc < __int_as_float(0x7f800000))) sc = 1.0f;
+        channel_body_clip(L, m, G, slice, sc, mode, qmax);
+    } else if (L.K > 1 && (mode & 6u) == 4u) {   // E + C without K
         channel_body_ec(L, m, G, slice, s, mode);
     } else if (L.K == 1) {
         if ((L.N & 3) == 0 && s >= 0x1p-60f && s <= 0x1p60f)

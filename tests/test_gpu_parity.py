@@ -388,3 +388,84 @@ def test_overlapping_calls_with_different_descriptors():
     for bufs, ws in ((ba, wa), (bb, wb)):
         for b, w in zip(bufs, ws):
             assert_layer_equal(b, w, 4, EKC)
+
+
+def _clip_scales(w, bits, lo=1.5, hi=4.0, seed=0):
+    """Per-channel scales 1.5 to 4 times smaller than the absmax scale (so that elements clip), with a
+    few special ones: the absmax scale itself, a far too large one, and invalid ones (-> 1)."""
+    m = w.shape[0]
+    qmax = 2 ** (bits - 1) - 1
+    a = np.abs(w.reshape(m, -1)).max(1)
+    a[a == 0] = 1.0
+    rng = np.random.default_rng(seed)
+    sc = (a / qmax / rng.uniform(lo, hi, size=m)).astype(np.float32)
+    sc[::5] = (a[::5] / np.float32(qmax)).astype(np.float32)
+    if m > 3:
+        sc[3] = np.float32(a[3] * 50)
+    if m > 7:
+        sc[6] = 0.0
+        sc[7] = np.nan
+    return sc
+
+
+@pytest.mark.parametrize("bits,flags", [(4, sq.FLAG_NARROW_RANGE), (3, 0), (8, sq.FLAG_NARROW_RANGE)])
+def test_caller_supplied_scales(bits, flags):
+    """Algorithm 1 with its scale as an input: the clip of Sec. 2.2 fires, clipped elements are
+    never flipped outward and kernels / channels can run out of candidates.  All kernel sizes, long
+    3x3 channels included (they leave the pipelined kernel), modes E, E|K, E|K|C and E|C on 1x1."""
+    shapes = [(12, 64, 3, 3), (9, 7, 3, 3), (10, 300, 1, 1), (6, 2049, 1, 1), (8, 5, 5, 5), (16, 1, 3, 3), (5, 3, 7, 7),
+              (4, 1024, 3, 3), (3, 33, 2, 2)]
+    ws = [W.random_layer(s, seed=300 + i) for i, s in enumerate(shapes)]
+    scs = [_clip_scales(w, bits, seed=i) for i, w in enumerate(ws)]
+    for mode in (EKC, EK, E):
+        bufs = [sq.alloc_outputs(torch.from_numpy(w).cuda()) for w in ws]
+        for b, sc in zip(bufs, scs):
+            b.scales_in = torch.from_numpy(sc).cuda()
+            b.codes.fill_(-128)
+        sq.squant_quantize_model(bufs, bits=bits, mode=mode, flags=flags)
+        sq.squant_device_status()
+        for b, w, sc, shp in zip(bufs, ws, scs, shapes):
+            r = oracle.quantize_layer(w, bits=bits, mode=mode, flags=flags, scales_in=sc)
+            assert np.array_equal(b.codes.cpu().numpy(), r.codes), f"{shp} mode {mode}"
+            assert np.array_equal(b.scales.cpu().numpy().view(np.uint32), r.scales.view(np.uint32))
+            assert np.array_equal(b.kernel_err.cpu().numpy().view(np.uint32), r.kernel_err.view(np.uint32)), f"{shp} mode {mode}"
+            assert np.array_equal(b.channel_err.cpu().numpy().view(np.uint32), r.channel_err.view(np.uint32)), f"{shp} mode {mode}"
+    # E|C: 1x1 layers only
+    mode = sq.MODE_E | sq.MODE_C
+    bufs = [sq.alloc_outputs(torch.from_numpy(ws[i]).cuda()) for i in (2, 3)]
+    for b, i in zip(bufs, (2, 3)):
+        b.scales_in = torch.from_numpy(scs[i]).cuda()
+    sq.squant_quantize_model(bufs, bits=bits, mode=mode, flags=flags)
+    sq.squant_device_status()
+    for b, i in zip(bufs, (2, 3)):
+        r = oracle.quantize_layer(ws[i], bits=bits, mode=mode, flags=flags, scales_in=scs[i])
+        assert np.array_equal(b.codes.cpu().numpy(), r.codes) and np.array_equal(b.channel_err.cpu().numpy(), r.channel_err)
+    b = sq.alloc_outputs(torch.from_numpy(ws[0]).cuda())
+    b.scales_in = torch.from_numpy(scs[0]).cuda()
+    with pytest.raises(sq.SquantError):
+        sq.squant_quantize_model([b], bits=bits, mode=mode, flags=flags)
+
+
+def test_caller_supplied_scales_other_outputs_and_host_path():
+    """Supplied scales with packed int4 and dequantized outputs, and through the host-buffer call."""
+    shapes = [(6, 64, 3, 3), (5, 256, 1, 1), (4, 3, 5, 5)]
+    ws = [W.random_layer(s, seed=340 + i) for i, s in enumerate(shapes)]
+    scs = [_clip_scales(w, 4, seed=20 + i) for i, w in enumerate(ws)]
+    flags = sq.FLAG_NARROW_RANGE | sq.FLAG_PACK_INT4
+    bufs = [sq.alloc_outputs(torch.from_numpy(w).cuda(), dequant=True, pack_int4=True) for w in ws]
+    for b, sc in zip(bufs, scs):
+        b.scales_in = torch.from_numpy(sc).cuda()
+    sq.squant_quantize_model(bufs, bits=4, flags=flags)
+    sq.squant_device_status()
+    for b, w, sc in zip(bufs, ws, scs):
+        r = oracle.quantize_layer(w, bits=4, flags=flags, scales_in=sc, details=True)
+        assert np.array_equal(b.codes.cpu().numpy(), r.codes)
+        assert np.array_equal(b.dequant.cpu().numpy().view(np.uint32), r.dequant.view(np.uint32))
+    hb = [sq.alloc_outputs(torch.from_numpy(w).pin_memory(), pin=True) for w in ws]
+    for b, sc in zip(hb, scs):
+        b.scales_in = torch.from_numpy(sc).pin_memory()
+    sq.squant_quantize_model_host(hb, bits=4)
+    for b, w, sc in zip(hb, ws, scs):
+        r = oracle.quantize_layer(w, bits=4, scales_in=sc)
+        assert np.array_equal(b.codes.numpy(), r.codes) and np.array_equal(b.kernel_err.numpy(), r.kernel_err)
+        assert np.array_equal(b.scales.numpy(), r.scales)
