@@ -68,6 +68,7 @@ extern "C" {
 #define SQUANT_ERR_NOMEM (-8)       /* host or device allocation failed */
 #define SQUANT_ERR_TIMEOUT (-10)    /* a kernel gave up a bounded wait on an asynchronous copy; the
                                        outputs of that launch are incomplete */
+#define SQUANT_ERR_CAPTURE (-11)    /* squant_quantize_layer_noalloc on a stream that is being captured */
 #define SQUANT_ERR_LIMIT (-9)       /* the layer needs more launch-table entries than the fixed
                                        table of squant_quantize_layer_noalloc holds */
 
@@ -187,7 +188,12 @@ int squant_plan_info(const squant_layer *layers, int32_t n_layers, const squant_
  * reading it.  Serialise such calls.
  *
  * The first call on each device looks up the table's device address and raises the kernel's
- * shared-memory limit; make that first call outside any stream capture.
+ * shared-memory limit; make that first call outside any stream capture.  Every call uploads the
+ * table from a host image inside the library that the next call rewrites, so a call on a stream
+ * that is being captured is refused (SQUANT_ERR_CAPTURE, nothing is enqueued).  The host image is
+ * ordinary pageable memory: the runtime stages such an upload through its own buffers, and the call
+ * can return only after that, which may mean waiting until earlier work on the stream has let the
+ * copy start - a caller in a latency-critical loop should count on the call blocking that long.
  *
  * Results are bit-identical to squant_quantize_layer.  Returns SQUANT_OK or a negative
  * SQUANT_ERR_* code; a failed call launches nothing and writes nothing.
@@ -219,6 +225,16 @@ int squant_selfcheck_division(const float *scales, int32_t n, int32_t bits, uint
  * SQUANT_ERR_TIMEOUT (and clears the record) or SQUANT_ERR_CUDA.
  */
 int squant_device_status(void);
+
+/*
+ * Test hooks for the failure path (no solver work).  squant_debug_set_status writes `value` into
+ * the device status word that squant_device_status reads, as a kernel that gave up a wait would.
+ * squant_debug_wait_expires launches one warp that waits, with a limit of max_polls (1..4096)
+ * polls, on a barrier nobody arrives at: the wait runs out, the kernel records it and ends - the
+ * next squant_device_status returns SQUANT_ERR_TIMEOUT and the context stays usable.
+ */
+int squant_debug_set_status(int value);
+int squant_debug_wait_expires(int32_t max_polls, void *cuda_stream);
 
 /* Number of kernels this library has launched in this process (all entry points). */
 int64_t squant_launch_count(void);

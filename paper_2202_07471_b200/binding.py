@@ -24,7 +24,7 @@ NOALLOC_MAX_CTAS = 32768
 
 EXPORTS = ("squant_quantize_layer", "squant_quantize_layer_noalloc", "squant_quantize_model", "squant_quantize_model_host",
            "squant_plan_info", "squant_selfcheck_division", "squant_device_status", "squant_launch_count", "squant_strerror", "squant_last_cuda_error",
-           "squant_shutdown")
+           "squant_shutdown", "squant_debug_set_status", "squant_debug_wait_expires")
 
 
 class SquantError(RuntimeError):
@@ -67,6 +67,10 @@ def load_library() -> ctypes.CDLL:
     for f in ("squant_quantize_layer", "squant_quantize_layer_noalloc", "squant_quantize_model", "squant_quantize_model_host",
               "squant_plan_info", "squant_selfcheck_division", "squant_device_status", "squant_shutdown"):
         getattr(lib, f).restype = ctypes.c_int
+    lib.squant_debug_set_status.argtypes = [ctypes.c_int]
+    lib.squant_debug_set_status.restype = ctypes.c_int
+    lib.squant_debug_wait_expires.argtypes = [ctypes.c_int32, vp]
+    lib.squant_debug_wait_expires.restype = ctypes.c_int
     lib.squant_launch_count.restype = ctypes.c_int64
     lib.squant_strerror.restype = ctypes.c_char_p
     lib.squant_strerror.argtypes = [ctypes.c_int]
@@ -236,6 +240,16 @@ def squant_selfcheck_division(scales, bits: int = 4):
 def squant_device_status() -> None:
     """Synchronise the current device; raise SquantError(-10) if a kernel gave up a bounded wait."""
     _check(load_library().squant_device_status())
+
+
+def squant_debug_set_status(value: int) -> None:
+    """Test hook: write the device status word as a kernel that gave up a wait would."""
+    _check(load_library().squant_debug_set_status(int(value)))
+
+
+def squant_debug_wait_expires(max_polls: int = 64, stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Test hook: one warp waits (at most max_polls polls) on a barrier nobody arrives at."""
+    _check(load_library().squant_debug_wait_expires(int(max_polls), _stream_handle(stream)))
 
 
 def squant_launch_count() -> int:

@@ -23,7 +23,7 @@ using sq::LayerDesc;
 constexpr int kMaxSmemFallback = 232448;   // 227 KB: per-CTA opt-in limit of sm_100
 constexpr int64_t kMaxChannelElems = 65535; // keeps the clamp-edge element out of every top-k
                                             // (its perturbation is <= one ulp of qmax)
-constexpr size_t kMaxPlans = 16;
+constexpr size_t kMaxPlans = 64;
 
 std::mutex g_mutex;
 std::atomic<int64_t> g_launches{0};
@@ -165,6 +165,7 @@ struct ParamPlan {
     // pipelined kernel (layers of long 3x3 channels): one item per output channel
     std::vector<sq::LaunchTable> pipe_tables;
     std::vector<int> pipe_items, pipe_set_stride, pipe_slot;
+    mutable bool slots_clean = false;   // the work counters of pipe_slot have been zeroed on the stream of the plan's first launch
 };
 
 int g_next_slot = 0;   // next work-counter slot of the pipelined kernel; guarded by g_mutex
@@ -334,8 +335,31 @@ int get_plan(const squant_layer *layers, int32_t n_layers, const squant_options 
     return SQUANT_OK;
 }
 
+// Device address of a work counter (done = false) or of its "CTAs finished" twin (done = true).
+void *ticket_address(int slot, bool done)
+{
+    static std::vector<std::pair<unsigned *, unsigned *>> base;   // per device; guarded by g_mutex
+    int device = 0;
+    cudaGetDevice(&device);
+    if (static_cast<int>(base.size()) <= device) base.resize(device + 1, {nullptr, nullptr});
+    if (!base[device].first) {
+        cudaGetSymbolAddress(reinterpret_cast<void **>(&base[device].first), sq::g_ticket);
+        cudaGetSymbolAddress(reinterpret_cast<void **>(&base[device].second), sq::g_done);
+    }
+    return (done ? base[device].second : base[device].first) + slot;
+}
+
 int launch_plan(const ParamPlan &p, cudaStream_t stream)
 {
+    // A work-counter slot comes to a plan in an unknown state (a plan that was evicted, or a launch
+    // that failed, may have left it dirty): zero it in stream order before the plan's first launch.
+    if (!p.slots_clean) {
+        for (size_t c = 0; c < p.pipe_tables.size(); ++c) {
+            SQ_CUDA(cudaMemsetAsync(ticket_address(p.pipe_slot[c], false), 0, sizeof(unsigned), stream));
+            SQ_CUDA(cudaMemsetAsync(ticket_address(p.pipe_slot[c], true), 0, sizeof(unsigned), stream));
+        }
+        p.slots_clean = true;
+    }
     // long 3x3 channels first: one persistent CTA per multiprocessor
     for (size_t c = 0; c < p.pipe_tables.size(); ++c) {
         if (p.pipe_items[c] == 0) continue;
@@ -558,6 +582,11 @@ int squant_quantize_layer_noalloc(const squant_layer *layer, const squant_option
     if (hp.items.size() > static_cast<size_t>(SQUANT_NOALLOC_MAX_CTAS)) return SQUANT_ERR_LIMIT;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     std::lock_guard<std::mutex> lock(g_mutex);
+    {   // the table upload below reads a host image that the next call rewrites: not for a captured stream
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        SQ_CUDA(cudaStreamIsCapturing(stream, &cap));
+        if (cap != cudaStreamCaptureStatusNone) return SQUANT_ERR_CAPTURE;
+    }
     int device = 0;
     SQ_CUDA(cudaGetDevice(&device));
     int limit = 0;
@@ -635,7 +664,26 @@ int squant_device_status(void)
     if (st == 0) return SQUANT_OK;
     const int zero = 0;
     SQ_CUDA(cudaMemcpyToSymbol(sq::g_device_status, &zero, sizeof(int)));
+    // a launch that gave up may have left its work counter half drawn: all plans start clean again
+    SQ_CUDA(cudaMemset(ticket_address(0, false), 0, sizeof(unsigned) * sq::kTicketSlots));
+    SQ_CUDA(cudaMemset(ticket_address(0, true), 0, sizeof(unsigned) * sq::kTicketSlots));
     return SQUANT_ERR_TIMEOUT;
+}
+
+int squant_debug_set_status(int value)
+{
+    std::lock_guard<std::mutex> lock(g_mutex);
+    SQ_CUDA(cudaMemcpyToSymbol(sq::g_device_status, &value, sizeof(int)));
+    return SQUANT_OK;
+}
+
+int squant_debug_wait_expires(int32_t max_polls, void *cuda_stream)
+{
+    if (max_polls < 1 || max_polls > 4096) return SQUANT_ERR_SHAPE;
+    sq::debug_wait_kernel<<<1, 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>(max_polls);
+    SQ_CUDA(cudaGetLastError());
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return SQUANT_OK;
 }
 
 int64_t squant_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
@@ -653,6 +701,7 @@ const char *squant_strerror(int code)
         case SQUANT_ERR_CUDA: return "a CUDA runtime call failed (see squant_last_cuda_error)";
         case SQUANT_ERR_NOMEM: return "out of host or device memory";
         case SQUANT_ERR_TIMEOUT: return "a kernel gave up a bounded wait on an asynchronous copy; outputs of that launch are incomplete";
+        case SQUANT_ERR_CAPTURE: return "squant_quantize_layer_noalloc was called on a stream that is being captured; it uploads its launch table from a host image that the next call rewrites";
         case SQUANT_ERR_LIMIT: return "the layer needs more thread blocks than the fixed launch table of squant_quantize_layer_noalloc holds (SQUANT_NOALLOC_MAX_CTAS); split it by output-channel range";
         default: return "unknown squant error code";
     }

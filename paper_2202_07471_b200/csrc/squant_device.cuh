@@ -103,10 +103,10 @@ __device__ __forceinline__ void mbar_arrive(void *bar)
 }
 
 // Bounded wait for phase `parity` of `bar`.  False if the limit ran out.
-__device__ __forceinline__ bool mbar_wait(void *bar, unsigned parity)
+__device__ __forceinline__ bool mbar_wait(void *bar, unsigned parity, int max_polls = kWaitIters)
 {
     const unsigned a = smem_addr(bar);
-    for (int it = 0; it < kWaitIters; ++it) {
+    for (int it = 0; it < max_polls; ++it) {
         unsigned done;
         asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
                      : "=r"(done) : "r"(a), "r"(parity) : "memory");
@@ -1368,6 +1368,18 @@ __global__ void selfcheck_division_kernel(const float *scales, int n, int qmax,
     }
     for (int o = 16; o > 0; o >>= 1) bad += __shfl_xor_sync(kFull, bad, o);
     if ((threadIdx.x & 31) == 0 && bad) atomicAdd(mismatches + si, bad);
+}
+
+// ---------------------------------------------------------------- the bounded wait, on its own
+// Waits for a barrier at which nobody ever arrives, with a small poll limit: the wait runs out,
+// the thread records it in the status word exactly as the solver kernels do, and the kernel ends.
+__global__ void debug_wait_kernel(int max_polls)
+{
+    __shared__ unsigned long long bar;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        if (!mbar_wait(&bar, 0u, max_polls)) atomicExch(&g_device_status, 1);
+    }
 }
 
 // ---------------------------------------------------------------- grouped launch

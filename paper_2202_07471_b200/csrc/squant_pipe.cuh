@@ -138,6 +138,7 @@ squant_pipe_kernel(const __grid_constant__ LaunchTable tbl, int qmax, unsigned m
     if (tid >= kPipeQuantThreads + kPipeFinThreads) {
         // ---------------------------------------------------------------- copy warp
         if (tid != kPipeQuantThreads + kPipeFinThreads) return;
+        int issued = 0;   // copies issued so far
         for (int i = 0;; ++i) {
             const int b = i & 1, u = i >> 1;
             int item = blockIdx.x;   // the grid never exceeds the number of items
@@ -155,6 +156,8 @@ squant_pipe_kernel(const __grid_constant__ LaunchTable tbl, int qmax, unsigned m
                 const int redo = reinterpret_cast<const volatile int *>(smem + static_cast<size_t>(b) * set_stride + red_off + 128)[6];
                 if (redo != 0) pipe_wait(ctrl, &ctrl->wfree[b], par);
             }
+            // after a wait of this CTA has run out, no further channel is started: the end mark goes out
+            if (*reinterpret_cast<volatile int *>(&ctrl->abort)) item = -1;
             ctrl->ring[b] = item;
             if (item < 0) {
                 mbar_arrive(&ctrl->full[b]);
@@ -165,6 +168,12 @@ squant_pipe_kernel(const __grid_constant__ LaunchTable tbl, int qmax, unsigned m
             const float *wg = L.w + static_cast<size_t>(item - tbl.first_item[layer]) * L.NK;
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the set's earlier readers before the async write
             bulk_load(smem + static_cast<size_t>(b) * set_stride, wg, static_cast<unsigned>(L.NK) * 4u, &ctrl->full[b]);
+            issued = i + 1;
+        }
+        if (*reinterpret_cast<volatile int *>(&ctrl->abort)) {
+            // leaving after a wait ran out: the last two copies may still be in flight into this
+            // CTA's shared memory; wait for them (bounded) before the CTA may end
+            for (int j = max(issued - 2, 0); j < issued; ++j) mbar_wait(&ctrl->full[j & 1], static_cast<unsigned>(j >> 1) & 1u);
         }
         // every ticket this CTA draws has been drawn: the last CTA to get here resets the slot
         __threadfence();

@@ -469,3 +469,25 @@ def test_caller_supplied_scales_other_outputs_and_host_path():
         r = oracle.quantize_layer(w, bits=4, scales_in=sc)
         assert np.array_equal(b.codes.numpy(), r.codes) and np.array_equal(b.kernel_err.numpy(), r.kernel_err)
         assert np.array_equal(b.scales.numpy(), r.scales)
+
+
+def test_failure_path_status_word_and_expiring_wait():
+    """Every wait inside the kernels is bounded; one that runs out sets a device status word that
+    squant_device_status reports once (SQUANT_ERR_TIMEOUT) and clears.  The plumbing is exercised
+    without disturbing any solver launch: by writing the word from the host, and by a one-warp
+    kernel whose wait on a barrier nobody arrives at runs out after 64 polls and returns.  The
+    context stays usable: a normal call afterwards matches the checker."""
+    sq.squant_device_status()                          # clean to start with
+    sq.squant_debug_set_status(1)
+    with pytest.raises(sq.SquantError) as ei:
+        sq.squant_device_status()
+    assert ei.value.code == -10
+    sq.squant_device_status()                          # reported once, then cleared
+    sq.squant_debug_wait_expires(64)
+    with pytest.raises(sq.SquantError) as ei:
+        sq.squant_device_status()
+    assert ei.value.code == -10
+    sq.squant_device_status()
+    w = W.random_layer((40, 1024, 3, 3), seed=12)      # pipelined kernel: its work counters were reset with the status
+    (b,) = run_gpu([w], 4, EKC)
+    assert_layer_equal(b, w, 4, EKC)

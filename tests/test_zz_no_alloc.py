@@ -9,9 +9,11 @@ Collected last on purpose (file name): a failure here cannot hide results of oth
 """
 import ctypes
 
+import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_2202_07471_b200 as sq
 from paper_2202_07471_b200 import binding, workloads as W
 
@@ -55,3 +57,30 @@ def test_noalloc_matches_regular_entry_point_on_consecutive_calls():
             torch.cuda.synchronize()
             assert sq.squant_launch_count() == n0 + 2
             assert _same(got, want), f"shape {shp} bits {bits}"
+            ref = oracle.quantize_layer(w.cpu().numpy(), bits=bits)      # and with the CPU checker directly
+            assert np.array_equal(got.codes.cpu().numpy(), ref.codes) and np.array_equal(got.scales.cpu().numpy(), ref.scales)
+            assert np.array_equal(got.kernel_err.cpu().numpy(), ref.kernel_err)
+            assert np.array_equal(got.channel_err.cpu().numpy(), ref.channel_err)
+
+
+@pytest.mark.gpu
+def test_noalloc_refuses_a_stream_that_is_being_captured():
+    """The table upload reads a host image that the next call rewrites, so a captured copy would
+    replay someone else's table: the call is refused before anything is enqueued, and the same
+    call works again on the same stream once the capture is over."""
+    w = torch.from_numpy(W.random_layer((32, 64, 3, 3), seed=5)).cuda()
+    got = sq.alloc_outputs(w)
+    sq.squant_quantize_layer_noalloc(got, bits=4)        # first call on the device: outside any capture
+    torch.cuda.synchronize()
+    want = got.codes.clone()
+    s = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
+    n0 = sq.squant_launch_count()
+    with torch.cuda.graph(g, stream=s):
+        with pytest.raises(sq.SquantError) as ei:
+            sq.squant_quantize_layer_noalloc(got, bits=4, stream=torch.cuda.current_stream())
+    assert ei.value.code == -11 and sq.squant_launch_count() == n0
+    got.codes.fill_(-128)
+    sq.squant_quantize_layer_noalloc(got, bits=4, stream=s)
+    s.synchronize()
+    assert torch.equal(got.codes, want)
