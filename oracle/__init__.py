@@ -37,7 +37,7 @@ def _load():
         lib.sqo_quantize_layer_scaled.argtypes = [
             ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
             ctypes.POINTER(_Options), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
-            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
         _lib = lib
     return _lib
 
@@ -51,6 +51,7 @@ class OracleResult:
     pert: Optional[np.ndarray] = None      # int32 fixed-point perturbations (2^-30 units)
     flip: Optional[np.ndarray] = None      # uint8: bit0 flipped by SQuant-K, bit1 by SQuant-C
     dequant: Optional[np.ndarray] = None   # fp32 code * scale (what Algorithm 1 returns)
+    dequant_bf16: Optional[np.ndarray] = None   # the same as bfloat16 bit patterns (uint16)
 
 
 def quantize_layer(w: np.ndarray, bits: int = 4, mode: int = MODE_EKC,
@@ -73,6 +74,7 @@ def quantize_layer(w: np.ndarray, bits: int = 4, mode: int = MODE_EKC,
     pert = np.empty(w.shape, dtype=np.int32) if details else None
     flip = np.empty(w.shape, dtype=np.uint8) if details else None
     deq = np.empty(w.shape, dtype=np.float32) if details else None
+    deq16 = np.empty(w.shape, dtype=np.uint16) if details else None
     opt = _Options(bits, mode, flags)
     ptr = lambda a: a.ctypes.data_as(ctypes.c_void_p) if a is not None else None
     sin = None
@@ -81,7 +83,7 @@ def quantize_layer(w: np.ndarray, bits: int = 4, mode: int = MODE_EKC,
         if sin.shape != (M,):
             raise ValueError("scales_in needs one fp32 scale per output channel")
     rc = _load().sqo_quantize_layer_scaled(ptr(w), M, N, K, ctypes.byref(opt), ptr(codes), ptr(scales),
-                                           ptr(kerr), ptr(cerr), ptr(pert), ptr(flip), ptr(deq), ptr(sin))
+                                           ptr(kerr), ptr(cerr), ptr(pert), ptr(flip), ptr(deq), ptr(sin), ptr(deq16))
     if rc != 0:
         raise ValueError(f"sqo_quantize_layer failed with code {rc}")
-    return OracleResult(codes, scales, kerr, cerr, pert, flip, deq)
+    return OracleResult(codes, scales, kerr, cerr, pert, flip, deq, deq16)

@@ -113,9 +113,18 @@ typedef struct {
     sqo_cand *list;  /* [N*K] scratch for sorting */
 } sqo_work;
 
+/* fp32 -> bfloat16 (the upper 16 bits of the fp32 pattern), round to nearest, ties to even. */
+static uint16_t sqo_bf16(float f)
+{
+    uint32_t u;
+    memcpy(&u, &f, sizeof(u));
+    u += 0x7fffu + ((u >> 16) & 1u);
+    return (uint16_t)(u >> 16);
+}
+
 static void sqo_channel(const float *w, int32_t N, int32_t K, const sqo_options *opt, const float *scale_in,
                         sqo_work *wk, int8_t *codes, float *scale_out,
-                        float *kernel_err, float *channel_err, float *dequant)
+                        float *kernel_err, float *channel_err, float *dequant, uint16_t *dequant_bf16)
 {
     const int32_t NK = N * K;
     const int32_t qmax = (1 << (opt->bits - 1)) - 1;
@@ -241,6 +250,8 @@ static void sqo_channel(const float *w, int32_t N, int32_t K, const sqo_options 
     if (channel_err) *channel_err = (float)total * 0x1p-30f;
     if (dequant)   /* what Algorithm 1 returns: C * s */
         for (int32_t j = 0; j < NK; ++j) dequant[j] = (float)q[j] * s;
+    if (dequant_bf16)   /* the same product (fp32), stored as bfloat16 */
+        for (int32_t j = 0; j < NK; ++j) dequant_bf16[j] = sqo_bf16((float)q[j] * s);
     if (opt->flags & SQO_FLAG_PACK_INT4) {
         for (int32_t j = 0; j < NK; j += 2) {
             unsigned lo = (unsigned)q[j] & 15u;
@@ -263,12 +274,14 @@ static void sqo_channel(const float *w, int32_t N, int32_t K, const sqo_options 
  *   flip         out [M][N][K] flip record (bit0 SQuant-K, bit1 SQuant-C), may be NULL
  *   dequant      out [M][N][K] fp32 code * scale (Algorithm 1's return value), may be NULL
  *   scales_in    in  [M] caller-supplied scales (Algorithm 1's input s), may be NULL: absmax scales
+ *   dequant_bf16 out [M][N][K] bfloat16 of the fp32 product code * scale (round to nearest even), may be NULL
  * pert is the perturbation clamped to 32 bits (exact whenever no element is clipped by more than
  * one step).  Inputs must be finite.  Returns SQO_OK or a negative error.
  */
 int sqo_quantize_layer_scaled(const float *w, int32_t M, int32_t N, int32_t K, const sqo_options *opt,
                               int8_t *codes, float *scales, float *kernel_err, float *channel_err,
-                              int32_t *pert, uint8_t *flip, float *dequant, const float *scales_in)
+                              int32_t *pert, uint8_t *flip, float *dequant, const float *scales_in,
+                              uint16_t *dequant_bf16)
 {
     if (!w || !opt || !codes || !scales || M < 0 || N <= 0 || K <= 0) return SQO_ERR_ARG;
     if (opt->bits < 2 || opt->bits > 8 || !(opt->mode & SQO_MODE_E)) return SQO_ERR_ARG;
@@ -291,7 +304,8 @@ int sqo_quantize_layer_scaled(const float *w, int32_t M, int32_t N, int32_t K, c
                         codes + (size_t)m * ((opt->flags & SQO_FLAG_PACK_INT4) ? (NK + 1) / 2 : NK), scales + m,
                         kernel_err ? kernel_err + (size_t)m * N : NULL,
                         channel_err ? channel_err + m : NULL,
-                        dequant ? dequant + (size_t)m * NK : NULL);
+                        dequant ? dequant + (size_t)m * NK : NULL,
+                        dequant_bf16 ? dequant_bf16 + (size_t)m * NK : NULL);
             if (pert)
                 for (size_t j = 0; j < NK; ++j) {
                     int64_t v = wk.P[j];
@@ -309,5 +323,5 @@ int sqo_quantize_layer(const float *w, int32_t M, int32_t N, int32_t K, const sq
                        int8_t *codes, float *scales, float *kernel_err, float *channel_err,
                        int32_t *pert, uint8_t *flip, float *dequant)
 {
-    return sqo_quantize_layer_scaled(w, M, N, K, opt, codes, scales, kernel_err, channel_err, pert, flip, dequant, NULL);
+    return sqo_quantize_layer_scaled(w, M, N, K, opt, codes, scales, kernel_err, channel_err, pert, flip, dequant, NULL, NULL);
 }

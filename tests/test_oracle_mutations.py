@@ -43,6 +43,7 @@ MUTATIONS = [
     ("scale denominator is qmax + 1", "s = (a < 0x1p-100f) ? 1.0f : a / (float)qmax;", "s = (a < 0x1p-100f) ? 1.0f : a / (float)(qmax + 1);"),
     ("supplied scale is ignored", "        s = *scale_in;", "        s = 1.0f; (void)scale_in;"),
     ("clip of Sec. 2.2 is missing at the upper bound", "        if (qf > (float)qmax) qf = (float)qmax;\n", ""),
+    ("bfloat16 output is truncated instead of rounded", "    u += 0x7fffu + ((u >> 16) & 1u);\n", ""),
     ("flip count is not limited by the candidates (SQuant-K)", "            int64_t k = sqo_flip_count(abs_e);\n            if (k > nc) k = nc;\n            for (int64_t r = 0; r < k; ++r) {\n                int32_t j = wk->list[r].idx;\n                q[j] -= sgn;\n                P[j] -= sgn * SQO_ONE;\n                wk->flip[j] |= 1;",
      "            int64_t k = sqo_flip_count(abs_e);\n            if (k > nc) k = nc > 0 ? nc - 1 : 0;\n            for (int64_t r = 0; r < k; ++r) {\n                int32_t j = wk->list[r].idx;\n                q[j] -= sgn;\n                P[j] -= sgn * SQO_ONE;\n                wk->flip[j] |= 1;"),
 ]
@@ -62,6 +63,7 @@ BATTERY = (
        lambda: props.test_squant_c_invariants((8, 16, 3, 3), 4, "coarse"),
        lambda: props.test_squant_c_invariants((2, 300, 1, 1), 8, "normal"),
        lambda: props.test_negation_scaling_permutation((8, 16, 3, 3), EKC),
+       lambda: props.test_dequantized_bf16_output_matches_the_library_conversion(4),
        scaled.test_hand_worked_clipped_kernel,
        scaled.test_hand_worked_clipped_channel,
        lambda: scaled.test_supplying_the_absmax_scale_changes_nothing(4, EKC),

@@ -420,3 +420,17 @@ def test_dequantized_output_is_code_times_scale(bits):
     err = np.abs(r.dequant.astype(np.float64) - w) / s
     assert err.max() < 1.0 + 1e-6
     assert err[r.flip == 0].max() <= 0.5 + 1e-6
+
+
+@pytest.mark.parametrize("bits", [2, 4, 8])
+def test_dequantized_bf16_output_matches_the_library_conversion(bits):
+    """Algorithm 1 returns C * s; as bfloat16 it is the fp32 product rounded to nearest even.
+    Cross-checked with PyTorch's own fp32 -> bfloat16 conversion (an independent routine)."""
+    import torch
+    w = _layer((6, 40, 3, 3), seed=30 + bits)
+    w[2] *= np.float32(2.0 ** 40)
+    w[3] *= np.float32(2.0 ** -40)
+    r = oracle.quantize_layer(w, bits=bits, details=True)
+    want = torch.from_numpy(r.dequant).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    assert np.array_equal(r.dequant_bf16, want)
+    assert (r.dequant_bf16 != (r.dequant.view(np.uint32) >> 16).astype(np.uint16)).any()   # rounding, not truncation, is exercised
