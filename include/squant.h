@@ -96,6 +96,8 @@ typedef struct squant_layer {
                                  perturbations */
     float *dequant;      /* out, may be NULL: [cout][cin][kh][kw] fp32 quantized weights
                                  code * s_m - what Algorithm 1 itself returns ("C * s") */
+    uint16_t *dequant_bf16; /* out, may be NULL: the same quantized weights as bfloat16 bit patterns
+                                 (the fp32 product code * s_m rounded to nearest, ties to even) */
     const float *scales_in; /* in, may be NULL: [cout] caller-supplied scales, the input s of
                                  Algorithm 1.  NULL: absmax scales (above).  With a supplied scale
                                  the clip of Sec. 2.2 really fires: a clipped element keeps its
@@ -118,7 +120,7 @@ int squant_quantize_layer(const squant_layer *layer, const squant_options *opt, 
  * Algorithm 1 on every layer of a model in one pass (the paper sums per-layer times and notes
  * that layers could be quantized in parallel, Sec. 4.2): ONE grouped kernel launch for all
  * layers, plus one launch of a pipelined kernel for those layers whose 3x3 output channels are
- * longer than 8192 weights (cin a multiple of 4 and at most 2048, SQuant-K on, int8 codes).
+ * longer than 8192 weights (cin a multiple of 4 and at most 2048, SQuant-K on, absmax scales).
  *
  *   layers, n_layers  host array of descriptors holding DEVICE pointers; n_layers >= 0
  *   opt               bits / mode / flags shared by all layers; NULL means 4 bit, E|K|C, narrow

@@ -41,7 +41,8 @@ class Layer(ctypes.Structure):
     _fields_ = [("w", ctypes.c_void_p), ("cout", ctypes.c_int32), ("cin", ctypes.c_int32),
                 ("kh", ctypes.c_int32), ("kw", ctypes.c_int32), ("codes", ctypes.c_void_p),
                 ("scales", ctypes.c_void_p), ("kernel_err", ctypes.c_void_p),
-                ("channel_err", ctypes.c_void_p), ("dequant", ctypes.c_void_p), ("scales_in", ctypes.c_void_p)]
+                ("channel_err", ctypes.c_void_p), ("dequant", ctypes.c_void_p), ("dequant_bf16", ctypes.c_void_p),
+                ("scales_in", ctypes.c_void_p)]
 
 
 _lib = None
@@ -97,10 +98,12 @@ class LayerBuffers:
     channel_err: Optional[torch.Tensor]
     dequant: Optional[torch.Tensor] = None     # fp32 code * scale, shape of the weights
     scales_in: Optional[torch.Tensor] = None   # fp32 [cout] caller-supplied scales (None: absmax scales)
+    dequant_bf16: Optional[torch.Tensor] = None   # bfloat16 code * scale, shape of the weights
 
 
 def alloc_outputs(w: torch.Tensor, kernel_err: bool = True, channel_err: bool = True,
-                  pin: bool = False, pack_int4: bool = False, dequant: bool = False) -> LayerBuffers:
+                  pin: bool = False, pack_int4: bool = False, dequant: bool = False,
+                  dequant_bf16: bool = False) -> LayerBuffers:
     """Allocate output tensors next to `w` ([cout, cin, kh, kw], [cout, cin, k] or [cout, cin]).
     With pack_int4 the codes tensor is [cout, ceil(cin*kh*kw / 2)] (for FLAG_PACK_INT4)."""
     if w.dtype != torch.float32 or not w.is_contiguous() or w.dim() < 2:
@@ -114,7 +117,8 @@ def alloc_outputs(w: torch.Tensor, kernel_err: bool = True, channel_err: bool = 
         w, torch.empty(cshape, dtype=torch.int8, **kw), torch.empty(m, dtype=torch.float32, **kw),
         torch.empty((m, n), dtype=torch.float32, **kw) if kernel_err else None,
         torch.empty(m, dtype=torch.float32, **kw) if channel_err else None,
-        torch.empty(w.shape, dtype=torch.float32, **kw) if dequant else None)
+        torch.empty(w.shape, dtype=torch.float32, **kw) if dequant else None, None,
+        torch.empty(w.shape, dtype=torch.bfloat16, **kw) if dequant_bf16 else None)
 
 
 def _descriptor(b: LayerBuffers) -> Layer:
@@ -133,7 +137,7 @@ def _descriptor(b: LayerBuffers) -> Layer:
                                     or b.scales_in.device != w.device):
         raise ValueError("scales_in must be a contiguous fp32 tensor [cout] next to the weights")
     return Layer(ptr(w), m, n, kh, kw, ptr(b.codes), ptr(b.scales), ptr(b.kernel_err), ptr(b.channel_err), ptr(b.dequant),
-                 ptr(b.scales_in))
+                 ptr(b.dequant_bf16), ptr(b.scales_in))
 
 
 def _options(bits: int, mode: int, flags: int) -> Options:
@@ -218,7 +222,7 @@ def squant_plan_info(shapes: Sequence[Sequence[int]], bits: int = 4, mode: int =
                      flags: int = FLAG_NARROW_RANGE) -> dict:
     """Launch geometry for layers of the given [cout, cin, kh, kw] shapes (no GPU needed)."""
     arr = (Layer * max(1, len(shapes)))(*[Layer(None, int(s[0]), int(s[1]), int(s[2]), int(s[3]),
-                                                None, None, None, None, None, None) for s in shapes])
+                                                None, None, None, None, None, None, None) for s in shapes])
     opt = _options(bits, mode, flags)
     g, t, s = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32()
     _check(load_library().squant_plan_info(arr, len(shapes), ctypes.byref(opt), ctypes.byref(g),

@@ -89,7 +89,7 @@ int validate(const squant_layer *layers, int32_t n_layers, const squant_options 
             if ((reinterpret_cast<uintptr_t>(l.w) & 3) || (reinterpret_cast<uintptr_t>(l.scales) & 3) ||
                 (reinterpret_cast<uintptr_t>(l.kernel_err) & 3) ||
                 (reinterpret_cast<uintptr_t>(l.channel_err) & 3) || (reinterpret_cast<uintptr_t>(l.dequant) & 3) ||
-                (reinterpret_cast<uintptr_t>(l.scales_in) & 3))
+                (reinterpret_cast<uintptr_t>(l.scales_in) & 3) || (reinterpret_cast<uintptr_t>(l.dequant_bf16) & 1))
                 return SQUANT_ERR_ALIGN;
         }
         // supplied scales: the element-wise channel step of E|C on larger kernels is not built for clipping
@@ -103,7 +103,7 @@ int validate(const squant_layer *layers, int32_t n_layers, const squant_options 
 int64_t layout_layer(const squant_layer &l, LayerDesc &d, unsigned mode)
 {
     d.w = l.w; d.codes = l.codes; d.scales = l.scales; d.kerr = l.kernel_err; d.cerr = l.channel_err; d.deq = l.dequant;
-    d.sin = l.scales_in;
+    d.sin = l.scales_in; d.deq16 = l.dequant_bf16;
     d.M = l.cout; d.N = l.cin; d.K = l.kh * l.kw; d.NK = d.N * d.K;
     d.g = group_size(d.NK);
     d.g_shift = 0;
@@ -171,12 +171,12 @@ struct ParamPlan {
 int g_next_slot = 0;   // next work-counter slot of the pipelined kernel; guarded by g_mutex
 
 // Layers the pipelined kernel takes: 3x3, more than 8192 weights per output channel (the grouped
-// kernel gives such a channel a whole CTA), input channels a multiple of four, SQuant-K on, plain
-// int8 codes, and two buffer sets fit the shared memory of one SM.
+// kernel gives such a channel a whole CTA), input channels a multiple of four, SQuant-K on, absmax
+// scales, and two buffer sets fit the shared memory of one SM.
 bool pipe_eligible(const squant_layer &l, const LayerDesc &d, const squant_options &o, int max_smem)
 {
     if (d.K != 9 || (d.N & 3) != 0 || d.NK <= 8192) return false;
-    if (!(o.mode & SQUANT_MODE_K) || (o.flags & SQUANT_FLAG_PACK_INT4) || l.dequant || l.scales_in) return false;
+    if (!(o.mode & SQUANT_MODE_K) || l.scales_in) return false;
     if ((reinterpret_cast<uintptr_t>(l.w) & 15) || (reinterpret_cast<uintptr_t>(l.codes) & 15)) return false;
     return 2 * d.slice_bytes + sq::kPipeCtrlBytes <= max_smem;
 }
@@ -476,20 +476,21 @@ int squant_quantize_model_host(const squant_layer *layers, int32_t n_layers,
     SQ_CUDA(cudaGetDevice(&device));
     // carve one device arena: per layer weights, codes, scales, kernel sums, channel sums
     std::vector<squant_layer> dev(layers, layers + n_layers);
-    std::vector<size_t> off(static_cast<size_t>(n_layers) * 7);
+    std::vector<size_t> off(static_cast<size_t>(n_layers) * 8);
     size_t total = 0;
     for (int i = 0; i < n_layers; ++i) {
         const squant_layer &l = layers[i];
         const size_t n = static_cast<size_t>(l.cin) * l.kh * l.kw * l.cout;
-        off[7 * i + 0] = total; total += align256(n * 4);
+        off[8 * i + 0] = total; total += align256(n * 4);
         const size_t code_bytes = (o.flags & SQUANT_FLAG_PACK_INT4)
                                       ? static_cast<size_t>(l.cout) * ((static_cast<size_t>(l.cin) * l.kh * l.kw + 1) / 2) : n;
-        off[7 * i + 1] = total; total += align256(code_bytes);
-        off[7 * i + 2] = total; total += align256(static_cast<size_t>(l.cout) * 4);
-        off[7 * i + 3] = total; total += l.kernel_err ? align256(static_cast<size_t>(l.cout) * l.cin * 4) : 0;
-        off[7 * i + 4] = total; total += l.channel_err ? align256(static_cast<size_t>(l.cout) * 4) : 0;
-        off[7 * i + 5] = total; total += l.dequant ? align256(n * 4) : 0;
-        off[7 * i + 6] = total; total += l.scales_in ? align256(static_cast<size_t>(l.cout) * 4) : 0;
+        off[8 * i + 1] = total; total += align256(code_bytes);
+        off[8 * i + 2] = total; total += align256(static_cast<size_t>(l.cout) * 4);
+        off[8 * i + 3] = total; total += l.kernel_err ? align256(static_cast<size_t>(l.cout) * l.cin * 4) : 0;
+        off[8 * i + 4] = total; total += l.channel_err ? align256(static_cast<size_t>(l.cout) * 4) : 0;
+        off[8 * i + 5] = total; total += l.dequant ? align256(n * 4) : 0;
+        off[8 * i + 6] = total; total += l.scales_in ? align256(static_cast<size_t>(l.cout) * 4) : 0;
+        off[8 * i + 7] = total; total += l.dequant_bf16 ? align256(n * 2) : 0;
     }
     if (static_cast<int>(g_arenas.size()) <= device) g_arenas.resize(device + 1);
     Arena &a = g_arenas[device];
@@ -502,13 +503,14 @@ int squant_quantize_model_host(const squant_layer *layers, int32_t n_layers,
     unsigned char *base = static_cast<unsigned char *>(a.ptr);
     for (int i = 0; i < n_layers; ++i) {
         const squant_layer &l = layers[i];
-        dev[i].w = reinterpret_cast<const float *>(base + off[7 * i + 0]);
-        dev[i].codes = reinterpret_cast<int8_t *>(base + off[7 * i + 1]);
-        dev[i].scales = reinterpret_cast<float *>(base + off[7 * i + 2]);
-        dev[i].kernel_err = l.kernel_err ? reinterpret_cast<float *>(base + off[7 * i + 3]) : nullptr;
-        dev[i].channel_err = l.channel_err ? reinterpret_cast<float *>(base + off[7 * i + 4]) : nullptr;
-        dev[i].dequant = l.dequant ? reinterpret_cast<float *>(base + off[7 * i + 5]) : nullptr;
-        dev[i].scales_in = l.scales_in ? reinterpret_cast<const float *>(base + off[7 * i + 6]) : nullptr;
+        dev[i].w = reinterpret_cast<const float *>(base + off[8 * i + 0]);
+        dev[i].codes = reinterpret_cast<int8_t *>(base + off[8 * i + 1]);
+        dev[i].scales = reinterpret_cast<float *>(base + off[8 * i + 2]);
+        dev[i].kernel_err = l.kernel_err ? reinterpret_cast<float *>(base + off[8 * i + 3]) : nullptr;
+        dev[i].channel_err = l.channel_err ? reinterpret_cast<float *>(base + off[8 * i + 4]) : nullptr;
+        dev[i].dequant = l.dequant ? reinterpret_cast<float *>(base + off[8 * i + 5]) : nullptr;
+        dev[i].scales_in = l.scales_in ? reinterpret_cast<const float *>(base + off[8 * i + 6]) : nullptr;
+        dev[i].dequant_bf16 = l.dequant_bf16 ? reinterpret_cast<uint16_t *>(base + off[8 * i + 7]) : nullptr;
     }
     // Chunks of consecutive layers (about kHostChunkBytes of weights each).  Uploads run on one
     // copy stream, each chunk's launches on the caller's stream once its upload is done, its
@@ -533,9 +535,9 @@ int squant_quantize_model_host(const squant_layer *layers, int32_t n_layers,
         for (int i = chunk_first[c]; i < chunk_first[c + 1]; ++i) {
             const squant_layer &l = layers[i];
             const size_t n = static_cast<size_t>(l.cin) * l.kh * l.kw * l.cout;
-            SQ_CUDA(cudaMemcpyAsync(base + off[7 * i + 0], l.w, n * 4, cudaMemcpyHostToDevice, hp->in));
+            SQ_CUDA(cudaMemcpyAsync(base + off[8 * i + 0], l.w, n * 4, cudaMemcpyHostToDevice, hp->in));
             if (l.scales_in)
-                SQ_CUDA(cudaMemcpyAsync(base + off[7 * i + 6], l.scales_in, static_cast<size_t>(l.cout) * 4, cudaMemcpyHostToDevice, hp->in));
+                SQ_CUDA(cudaMemcpyAsync(base + off[8 * i + 6], l.scales_in, static_cast<size_t>(l.cout) * 4, cudaMemcpyHostToDevice, hp->in));
         }
         SQ_CUDA(cudaEventRecord(hp->uploaded[c], hp->in));
     }
@@ -562,6 +564,8 @@ int squant_quantize_model_host(const squant_layer *layers, int32_t n_layers,
                 SQ_CUDA(cudaMemcpyAsync(l.channel_err, dev[i].channel_err, static_cast<size_t>(l.cout) * 4, cudaMemcpyDeviceToHost, hp->out));
             if (l.dequant)
                 SQ_CUDA(cudaMemcpyAsync(l.dequant, dev[i].dequant, n * 4, cudaMemcpyDeviceToHost, hp->out));
+            if (l.dequant_bf16)
+                SQ_CUDA(cudaMemcpyAsync(l.dequant_bf16, dev[i].dequant_bf16, n * 2, cudaMemcpyDeviceToHost, hp->out));
         }
     }
     SQ_CUDA(cudaStreamSynchronize(hp->out));

@@ -31,6 +31,7 @@ struct LayerDesc {
     float *cerr;
     float *deq;
     const float *sin;     // caller-supplied scales, or null: absmax scales
+    uint16_t *deq16;      // bfloat16 code * s, or null
     int32_t M, N, K, NK;
     int32_t g;            // threads per channel group: 32, 64, 128 or 256
     int32_t g_shift;      // log2(g)
@@ -705,11 +706,34 @@ __device__ __forceinline__ ChannelStep channel_step(const LayerDesc &L, const Gr
 constexpr unsigned kModePackInt4 = 0x100u;
 constexpr unsigned kModeWideRange = 0x200u;   // the clip range is [-qmax - 1, qmax] (no narrow-range flag)
 
+// fp32 -> bfloat16 (the upper half of the fp32 pattern), round to nearest, ties to even; finite input
+__device__ __forceinline__ unsigned bf16_bits(float f)
+{
+    const unsigned u = __float_as_uint(f);
+    return (u + 0x7fffu + ((u >> 16) & 1u)) >> 16;
+}
+
 __device__ __forceinline__ void emit_channel(const LayerDesc &L, int m, const Group &G,
                                              const unsigned char *cbuf, unsigned char *scratch, float s,
                                              long long ec, unsigned mode)
 {
     const int NK = L.NK;
+    if (L.deq16) {   // the same product as bfloat16
+        uint16_t *dg = L.deq16 + static_cast<size_t>(m) * NK;
+        if ((reinterpret_cast<uintptr_t>(dg) & 7) == 0 && (NK & 3) == 0) {
+            for (int i = G.t; i < (NK >> 2); i += G.g) {
+                const unsigned c4 = reinterpret_cast<const unsigned *>(cbuf)[i];
+                const unsigned b0 = bf16_bits(__fmul_rn(__int2float_rn(static_cast<signed char>(c4 & 255u)), s));
+                const unsigned b1 = bf16_bits(__fmul_rn(__int2float_rn(static_cast<signed char>((c4 >> 8) & 255u)), s));
+                const unsigned b2 = bf16_bits(__fmul_rn(__int2float_rn(static_cast<signed char>((c4 >> 16) & 255u)), s));
+                const unsigned b3 = bf16_bits(__fmul_rn(__int2float_rn(static_cast<signed char>(c4 >> 24)), s));
+                __stcs(reinterpret_cast<uint2 *>(dg) + i, make_uint2(b0 | (b1 << 16), b2 | (b3 << 16)));
+            }
+        } else {
+            for (int i = G.t; i < NK; i += G.g)
+                dg[i] = static_cast<uint16_t>(bf16_bits(__fmul_rn(__int2float_rn(static_cast<signed char>(cbuf[i])), s)));
+        }
+    }
     if (L.deq) {   // Algorithm 1's own return value: code * s, fp32
         float *dg = L.deq + static_cast<size_t>(m) * NK;
         if ((reinterpret_cast<uintptr_t>(dg) & 15) == 0 && (NK & 3) == 0) {
@@ -989,7 +1013,7 @@ template <int KT>
 __device__ __forceinline__ void finish_channel_hist(const LayerDesc &L, int m, const Group &G,
                                                     unsigned char *slice, float s, unsigned mode,
                                                     long long esum, float *kerr, float y, float s2,
-                                                    void *w_release = nullptr)
+                                                    void *w_release = nullptr, unsigned char *pack_scratch = nullptr)
 {
     const int N = L.N;
     unsigned char *cbuf = slice + L.off_codes;
@@ -1154,7 +1178,7 @@ __device__ __forceinline__ void finish_channel_hist(const LayerDesc &L, int m, c
     }
 
     // ---- codes, scale, channel error (the staged weights / perturbations are dead: scratch)
-    emit_channel(L, m, G, cbuf, slice, s, ec, mode);
+    emit_channel(L, m, G, cbuf, pack_scratch ? pack_scratch : slice, s, ec, mode);
 }
 
 // ---------------------------------------------------------------- channel body, 3x3 fast path

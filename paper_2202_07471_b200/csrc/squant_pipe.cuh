@@ -106,7 +106,7 @@ __device__ __forceinline__ long long k9_quantize_div(const LayerDesc &L, int m, 
     return esum;
 }
 
-// Layers: 3x3, N a multiple of 4, SQuant-K on, no packed and no dequantized output; every layer
+// Layers: 3x3, N a multiple of 4, SQuant-K on; every layer
 // descriptor carries the 512-thread layout of the grouped kernel, and a buffer set is one such
 // slice (set_stride bytes apart).  One item = one output channel.
 __global__ void __launch_bounds__(kPipeThreads, 1)
@@ -267,7 +267,9 @@ squant_pipe_kernel(const __grid_constant__ LaunchTable tbl, int qmax, unsigned m
         const float s2 = __fmul_rn(s, 0x1p-30f);
         const float y = __frcp_rn(s2);   // only the exact redo uses it (fast-path channels)
         float *kerr = L.kerr ? L.kerr + static_cast<size_t>(m) * L.N : nullptr;
-        finish_channel_hist<9>(L, m, G, slice, s, mode, 0ll, kerr, y, s2, &ctrl->wfree[b]);
+        // packed rows are put together in the set's candidate arrays (dead by then): the staged
+        // weights' place may already be receiving the set's next channel
+        finish_channel_hist<9>(L, m, G, slice, s, mode, 0ll, kerr, y, s2, &ctrl->wfree[b], slice + L.off_ev);
         G.sync();   // every finisher is done with the set; the first one has waited for its bulk store
         {   // leave the channel-step scratch cleared for the set's next channel
             int *scratch = reinterpret_cast<int *>(slice + hist_off);

@@ -70,13 +70,13 @@ def test_valid_edge_arguments():
 
 def test_null_pointers_are_rejected_before_any_cuda_call():
     lib = sq.load_library()
-    layer = binding.Layer(None, 4, 3, 3, 3, None, None, None, None, None, None)
+    layer = binding.Layer(None, 4, 3, 3, 3, None, None, None, None, None, None, None)
     opt = binding.Options(4, 7, 1)
     assert lib.squant_quantize_layer(ctypes.byref(layer), ctypes.byref(opt), None) == -1
     assert lib.squant_quantize_model(None, 2, ctypes.byref(opt), None) == -1
     assert lib.squant_quantize_model(None, 0, ctypes.byref(opt), None) == 0
     assert lib.squant_quantize_layer(None, ctypes.byref(opt), None) == -1
-    layer = binding.Layer(1026, 4, 3, 3, 3, 64, 128, None, None, None, None)      # weights not 4-byte aligned
+    layer = binding.Layer(1026, 4, 3, 3, 3, 64, 128, None, None, None, None, None)      # weights not 4-byte aligned
     assert lib.squant_quantize_layer(ctypes.byref(layer), ctypes.byref(opt), None) == -5
 
 

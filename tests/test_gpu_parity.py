@@ -311,19 +311,32 @@ def test_boundary_bin_between_list_and_radix_capacity(k):
 
 
 def test_dequantized_output():
-    """Optional fp32 output code * s (what Algorithm 1 returns), all paths, aligned and not."""
-    shapes = [(6, 64, 3, 3), (3, 2048, 3, 3), (5, 256, 1, 1), (7, 33, 1, 1), (4, 3, 5, 5), (3, 7, 3, 3)]
+    """Optional outputs code * s (what Algorithm 1 returns) in fp32 and bfloat16, all paths - the
+    pipelined kernel for the long 3x3 channels included -, aligned and not, with int8 and packed codes."""
+    shapes = [(6, 64, 3, 3), (3, 2048, 3, 3), (150, 1000, 3, 3), (5, 256, 1, 1), (7, 33, 1, 1), (4, 3, 5, 5), (3, 7, 3, 3)]
     ws = [adversarial_layer(s, seed=40 + i) for i, s in enumerate(shapes)]
     for flags, pack in ((sq.FLAG_NARROW_RANGE, False), (sq.FLAG_NARROW_RANGE | sq.FLAG_PACK_INT4, True)):
-        bufs = [sq.alloc_outputs(torch.from_numpy(w).cuda(), dequant=True, pack_int4=pack) for w in ws]
+        bufs = [sq.alloc_outputs(torch.from_numpy(w).cuda(), dequant=True, pack_int4=pack, dequant_bf16=True) for w in ws]
         for b in bufs:
             b.dequant.fill_(float("nan"))
+            b.dequant_bf16.fill_(float("nan"))
         sq.squant_quantize_model(bufs, bits=4, mode=EKC, flags=flags)
         sq.squant_device_status()
         for b, w, shp in zip(bufs, ws, shapes):
             r = oracle.quantize_layer(w, bits=4, mode=EKC, flags=flags, details=True)
             assert np.array_equal(b.dequant.cpu().numpy().view(np.uint32), r.dequant.view(np.uint32)), f"shape {shp}"
-            assert np.array_equal(b.codes.cpu().numpy(), r.codes)
+            assert np.array_equal(b.dequant_bf16.view(torch.int16).cpu().numpy().view(np.uint16), r.dequant_bf16), f"shape {shp}"
+            assert np.array_equal(b.codes.cpu().numpy(), r.codes), f"shape {shp}"
+            assert np.array_equal(b.kernel_err.cpu().numpy().view(np.uint32), r.kernel_err.view(np.uint32))
+    # bfloat16 alone, on a view that starts off an 8-byte boundary
+    w = ws[0]
+    base = torch.zeros(w.size + 1, dtype=torch.bfloat16, device="cuda")
+    b = sq.alloc_outputs(torch.from_numpy(w).cuda())
+    b.dequant_bf16 = base[1:].view(w.shape)
+    sq.squant_quantize_model([b], bits=4)
+    sq.squant_device_status()
+    r = oracle.quantize_layer(w, bits=4, details=True)
+    assert np.array_equal(b.dequant_bf16.contiguous().view(torch.int16).cpu().numpy().view(np.uint16), r.dequant_bf16)
 
 
 def test_host_entry_point_several_chunks_against_the_checker():

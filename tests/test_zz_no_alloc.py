@@ -23,7 +23,7 @@ def test_layer_beyond_the_fixed_table_is_rejected_without_a_gpu():
     lib = sq.load_library()
     m = sq.NOALLOC_MAX_CTAS + 1                      # channels of 18432 weights: one block each
     assert sq.squant_plan_info([(m, 2048, 3, 3)])["grid_ctas"] == m
-    layer = binding.Layer(256, m, 2048, 3, 3, 256, 256, None, None, None, None)   # never dereferenced
+    layer = binding.Layer(256, m, 2048, 3, 3, 256, 256, None, None, None, None, None)   # never dereferenced
     opt = binding.Options(4, sq.MODE_EKC, sq.FLAG_NARROW_RANGE)
     rc = lib.squant_quantize_layer_noalloc(ctypes.byref(layer), ctypes.byref(opt), None)
     assert rc == -9
