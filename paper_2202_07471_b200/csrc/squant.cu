@@ -14,6 +14,7 @@
 
 #include "squant_device.cuh"
 #include "squant_pipe.cuh"
+#include "squant_wide.cuh"
 
 namespace {
 
@@ -21,8 +22,10 @@ using sq::Item;
 using sq::LayerDesc;
 
 constexpr int kMaxSmemFallback = 232448;   // 227 KB: per-CTA opt-in limit of sm_100
-constexpr int64_t kMaxChannelElems = 65535; // keeps the clamp-edge element out of every top-k
-                                            // (its perturbation is <= one ulp of qmax)
+constexpr int64_t kMaxChannelElems = 65535; // one-CTA paths: keeps the clamp-edge element out of every top-k (its
+                                            // perturbation is <= one ulp of qmax); wider channels take the cluster
+                                            // kernel, which checks every candidate against the clip range
+constexpr int64_t kMaxKernels = (1 << sq::kIdxBits) - 1;   // kernels per channel: the select keys hold 18 index bits
 constexpr size_t kMaxPlans = 64;
 
 std::mutex g_mutex;
@@ -83,7 +86,7 @@ int validate(const squant_layer *layers, int32_t n_layers, const squant_options 
         const int64_t nk = k * l.cin;
         if (k > 65535 || nk > (1ll << 30)) return SQUANT_ERR_SHAPE;
         if (static_cast<int64_t>(l.cout) * nk > (1ll << 40)) return SQUANT_ERR_SHAPE;
-        if (nk > kMaxChannelElems) return SQUANT_ERR_TOO_WIDE;
+        if (l.cin > kMaxKernels) return SQUANT_ERR_TOO_WIDE;
         if (need_pointers) {
             if (!l.w || !l.codes || !l.scales) return SQUANT_ERR_NULL;
             if ((reinterpret_cast<uintptr_t>(l.w) & 3) || (reinterpret_cast<uintptr_t>(l.scales) & 3) ||
@@ -162,6 +165,9 @@ struct ParamPlan {
     std::vector<int> grids;
     int smem_bytes = 0, qmax = 0;
     unsigned mode = 0;
+    // cluster kernel (channels wider than one CTA): one launch per layer
+    struct Wide { LayerDesc d; int cluster, kpc, smem; };
+    std::vector<Wide> wide;
     // pipelined kernel (layers of long 3x3 channels): one item per output channel
     std::vector<sq::LaunchTable> pipe_tables;
     std::vector<int> pipe_items, pipe_set_stride, pipe_slot;
@@ -192,7 +198,19 @@ int build_param_plan(const squant_layer *layers, int32_t n_layers, const squant_
     std::vector<int> order, piped;
     for (int i = 0; i < n_layers; ++i) {
         const int64_t cta_smem = layout_layer(layers[i], descs[i], o.mode);
-        if (cta_smem > max_smem) return SQUANT_ERR_TOO_WIDE;
+        if (cta_smem > max_smem || descs[i].NK > kMaxChannelElems) {
+            // a cluster of 2, 4 or 8 CTAs per output channel, each with an even number of kernels
+            if ((o.mode & SQUANT_MODE_C) && !(o.mode & SQUANT_MODE_K) && descs[i].K > 1) return SQUANT_ERR_TOO_WIDE;   // E|C selects among elements: one CTA only
+            ParamPlan::Wide w{descs[i], 0, 0, 0};
+            for (int c = 2; c <= sq::kWideMaxCluster && !w.cluster; c *= 2) {
+                const int kpc = (((descs[i].N + c - 1) / c) + 1) & ~1;
+                const sq::WideLayout wl = sq::wide_layout(kpc, descs[i].K);
+                if (wl.total <= max_smem) { w.cluster = c; w.kpc = kpc; w.smem = wl.total; }
+            }
+            if (!w.cluster) return SQUANT_ERR_TOO_WIDE;
+            p.wide.push_back(w);
+            continue;
+        }
         if (pipe_eligible(layers[i], descs[i], o, max_smem)) {
             piped.push_back(i);
             continue;
@@ -299,6 +317,8 @@ int device_smem_limit(int device, int &limit)
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, v));
         SQ_CUDA(cudaFuncSetAttribute(sq::squant_pipe_kernel,
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, v));
+        SQ_CUDA(cudaFuncSetAttribute(sq::squant_wide_kernel,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, v));
         int sms = 0;
         SQ_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
         if (static_cast<int>(g_sm_count_by_device.size()) <= device) g_sm_count_by_device.resize(device + 1, 0);
@@ -376,6 +396,22 @@ int launch_plan(const ParamPlan &p, cudaStream_t stream)
         if (p.grids[c] == 0) continue;
         sq::squant_model_kernel<<<p.grids[c], sq::kCtaThreads, p.smem_bytes, stream>>>(p.tables[c], p.qmax, p.mode);
         SQ_CUDA(cudaGetLastError());
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+    }
+    for (const ParamPlan::Wide &w : p.wide) {   // one cluster per output channel
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(static_cast<unsigned>(w.d.M) * w.cluster);
+        cfg.blockDim = dim3(sq::kWideThreads);
+        cfg.dynamicSmemBytes = static_cast<size_t>(w.smem);
+        cfg.stream = stream;
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributeClusterDimension;
+        attr.val.clusterDim.x = static_cast<unsigned>(w.cluster);
+        attr.val.clusterDim.y = 1;
+        attr.val.clusterDim.z = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        SQ_CUDA(cudaLaunchKernelEx(&cfg, sq::squant_wide_kernel, w.d, p.qmax, p.mode, w.kpc));
         g_launches.fetch_add(1, std::memory_order_relaxed);
     }
     return SQUANT_OK;
@@ -701,7 +737,7 @@ const char *squant_strerror(int code)
         case SQUANT_ERR_BITS: return "bits must be in 2..8 (2..4 with SQUANT_FLAG_PACK_INT4)";
         case SQUANT_ERR_MODE: return "mode mask must contain E (E, E|K, E|C or E|K|C); unknown mode or flag bits are rejected";
         case SQUANT_ERR_ALIGN: return "float pointers must be 4-byte aligned";
-        case SQUANT_ERR_TOO_WIDE: return "an output channel (cin*kh*kw) does not fit the on-chip path";
+        case SQUANT_ERR_TOO_WIDE: return "an output channel (cin*kh*kw) does not fit the on-chip path, not even spread over a cluster of 8 thread blocks";
         case SQUANT_ERR_CUDA: return "a CUDA runtime call failed (see squant_last_cuda_error)";
         case SQUANT_ERR_NOMEM: return "out of host or device memory";
         case SQUANT_ERR_TIMEOUT: return "a kernel gave up a bounded wait on an asynchronous copy; outputs of that launch are incomplete";

@@ -859,6 +859,57 @@ __device__ __forceinline__ void channel_body(const LayerDesc &L, int m, const Gr
 // out of candidates before its sum is within one half.  Plain thread-per-kernel code, any kernel
 // size, IEEE division; correctness first.  The layer's slice keeps e', v and idx in arrays of
 // their own also for 1x1 kernels (the host lays such layers out that way).
+// SQuant-E with the clip, SQuant-K with in-range flips only and the candidate of Algorithm 3 for
+// the kernel whose K weights sit at wk (overwritten by the 32-bit perturbations); codes go to ck.
+__device__ __forceinline__ void kernel_clip(float *wk, int K, float s, bool do_k, int qmin, int qmax, int8_t *ck,
+                                            long long &e_out, int &v_out, int &idx_out)
+{
+    int *Pk = reinterpret_cast<int *>(wk);
+    long long e = 0;
+    for (int i = 0; i < K; ++i) {
+        const float x = __fdiv_rn(wk[i], s);
+        const float qf = fminf(fmaxf(rintf(x), static_cast<float>(qmin)), static_cast<float>(qmax));   // the clip of Sec. 2.2
+        const long long P = __float2ll_rn(__fmul_rn(__fsub_rn(qf, x), 1073741824.0f));
+        ck[i] = static_cast<int8_t>(__float2int_rn(qf));
+        Pk[i] = static_cast<int>(max(min(P, 0x7fffffffll), -0x7fffffffll));
+        e += P;
+    }
+    int v = 0, idx = 0;
+    if (e != 0) {
+        const int sgn = e > 0 ? 1 : -1;
+        const long long abs_e = e > 0 ? e : -e;
+        const int k = do_k ? static_cast<int>(min((abs_e + (kHalf - 1)) >> 30, static_cast<long long>(K) + 1)) : 0;
+        int flips = 0, last = -1, cand = -1;
+        for (int r = 0; r <= k; ++r) {
+            int best = 0, bi = -1;
+            for (int i = 0; i < K; ++i) {
+                const int key = sgn * Pk[i], fl = ck[i] - sgn;
+                if (key > best && fl >= qmin && fl <= qmax) { best = key; bi = i; }
+            }
+            if (bi < 0) break;   // out of candidates: the kernel keeps what is left of its sum
+            if (r < k) {
+                Pk[bi] -= sgn * kOne;
+                ck[bi] = static_cast<int8_t>(ck[bi] - sgn);
+                last = bi;
+                ++flips;
+            } else {
+                cand = bi;
+            }
+        }
+        e -= static_cast<long long>(sgn) * flips * kOne;
+        if (static_cast<long long>(flips) * kOne > abs_e) {   // Over SQuant: flip back candidate
+            idx = last;
+            v = Pk[last];
+        } else if (cand >= 0) {                               // Under SQuant: next un-flipped
+            idx = cand;
+            v = Pk[cand];
+        }
+    }
+    e_out = e;
+    v_out = v;
+    idx_out = idx;
+}
+
 __device__ __forceinline__ void channel_body_clip(const LayerDesc &L, int m, const Group &G, unsigned char *slice, float s,
                                                   unsigned mode, int qmax)
 {
@@ -873,49 +924,9 @@ __device__ __forceinline__ void channel_body_clip(const LayerDesc &L, int m, con
     float *kerr = L.kerr ? L.kerr + static_cast<size_t>(m) * N : nullptr;
     long long esum = 0;
     for (int n = G.t; n < N; n += G.g) {
-        float *wk = wbuf + static_cast<size_t>(n) * K;
-        int *Pk = reinterpret_cast<int *>(wk);   // the 32-bit perturbations overwrite the weights
-        int8_t *ck = cbuf + static_cast<size_t>(n) * K;
-        long long e = 0;
-        for (int i = 0; i < K; ++i) {
-            const float x = __fdiv_rn(wk[i], s);
-            const float qf = fminf(fmaxf(rintf(x), static_cast<float>(qmin)), static_cast<float>(qmax));   // the clip of Sec. 2.2
-            const long long P = __float2ll_rn(__fmul_rn(__fsub_rn(qf, x), 1073741824.0f));
-            ck[i] = static_cast<int8_t>(__float2int_rn(qf));
-            Pk[i] = static_cast<int>(max(min(P, 0x7fffffffll), -0x7fffffffll));
-            e += P;
-        }
-        int v = 0, idx = 0;
-        if (e != 0) {
-            const int sgn = e > 0 ? 1 : -1;
-            const long long abs_e = e > 0 ? e : -e;
-            const int k = do_k ? static_cast<int>(min((abs_e + (kHalf - 1)) >> 30, static_cast<long long>(K) + 1)) : 0;
-            int flips = 0, last = -1, cand = -1;
-            for (int r = 0; r <= k; ++r) {
-                int best = 0, bi = -1;
-                for (int i = 0; i < K; ++i) {
-                    const int key = sgn * Pk[i], fl = ck[i] - sgn;
-                    if (key > best && fl >= qmin && fl <= qmax) { best = key; bi = i; }
-                }
-                if (bi < 0) break;   // out of candidates: the kernel keeps what is left of its sum
-                if (r < k) {
-                    Pk[bi] -= sgn * kOne;
-                    ck[bi] = static_cast<int8_t>(ck[bi] - sgn);
-                    last = bi;
-                    ++flips;
-                } else {
-                    cand = bi;
-                }
-            }
-            e -= static_cast<long long>(sgn) * flips * kOne;
-            if (static_cast<long long>(flips) * kOne > abs_e) {   // Over SQuant: flip back candidate
-                idx = last;
-                v = Pk[last];
-            } else if (cand >= 0) {                               // Under SQuant: next un-flipped
-                idx = cand;
-                v = Pk[cand];
-            }
-        }
+        long long e;
+        int v, idx;
+        kernel_clip(wbuf + static_cast<size_t>(n) * K, K, s, do_k, qmin, qmax, cbuf + static_cast<size_t>(n) * K, e, v, idx);
         // a kernel that SQuant-C can flip has a candidate, hence |e'| <= 1/2: its 32-bit copy is exact
         ev[n] = static_cast<int>(max(min(e, 0x7fffffffll), -0x7fffffffll));
         vv[n] = v;

@@ -504,3 +504,62 @@ def test_failure_path_status_word_and_expiring_wait():
     w = W.random_layer((40, 1024, 3, 3), seed=12)      # pipelined kernel: its work counters were reset with the status
     (b,) = run_gpu([w], 4, EKC)
     assert_layer_equal(b, w, 4, EKC)
+
+
+def _edge_scale_case(n):
+    """One channel of n 1x1 kernels in which the absmax element lands a shade above qmax (its flip
+    would leave the range) and every other element ties with it in perturbation: SQuant-C must
+    skip the edge element although it comes first in the tie order."""
+    qmax = np.float32(127.0)
+    a = None
+    for t in np.linspace(1.0, 2.0, 4000, dtype=np.float32):
+        if np.float32(t) / (np.float32(t) / qmax) > qmax:
+            a = np.float32(t)
+            break
+    assert a is not None
+    s = a / qmax
+    w = np.full((1, n, 1, 1), s * np.float32(2.0 ** -17), dtype=np.float32)
+    w[0, 0, 0, 0] = a
+    return w
+
+
+def test_channels_wider_than_one_thread_block():
+    """Channels that do not fit one thread block's shared memory take the cluster kernel (2 to 8
+    blocks per output channel, absmax / channel sum / select histograms exchanged through
+    distributed shared memory).  Fully connected layers of 100,000 and 262,143 inputs, 3x3 and 5x5
+    layers with 8192 and 2600 kernels per channel, every mode, special channels; and the case in
+    which the range exclusion binds (70,000 tied candidates, the first of them on the clip edge)."""
+    shapes = [(3, 100000, 1, 1), (2, 8192, 3, 3), (2, 2600, 5, 5), (2, 262143, 1, 1), (9, 46001, 1, 1), (3, 4100, 3, 3)]
+    ws = [adversarial_layer(s, seed=500 + i) for i, s in enumerate(shapes)]
+    n0 = sq.squant_launch_count()
+    for bits, mode in ((4, EKC), (8, EK), (3, E)):
+        bufs = run_gpu(ws, bits, mode)
+        for b, w, shp in zip(bufs, ws, shapes):
+            assert_layer_equal(b, w, bits, mode, tag=f"{shp} bits {bits} mode {mode}")
+    assert sq.squant_launch_count() == n0 + 3 * (4 + 1)   # one cluster launch per wide layer; the last two shapes still fit one block
+    w = _edge_scale_case(70000)
+    for mode in (EKC, sq.MODE_E | sq.MODE_C):
+        (b,) = run_gpu([w], 8, mode)
+        r = oracle.quantize_layer(w, bits=8, mode=mode, details=True)
+        assert r.codes[0, 0, 0, 0] == 127 and r.codes[0, 1, 0, 0] == 1 and int(r.codes[0, 2:].max()) == 0   # the checker skipped the edge element
+        assert_layer_equal(b, w, 8, mode, tag=f"edge case mode {mode}")
+    # a wide layer next to ordinary ones in one call; packed and dequantized outputs; supplied scales
+    ws2 = [W.random_layer((4, 64, 3, 3), seed=1), W.random_layer((2, 70001, 1, 1), seed=2), W.random_layer((3, 9000, 3, 3), seed=3)]
+    flags = sq.FLAG_NARROW_RANGE | sq.FLAG_PACK_INT4
+    bufs = [sq.alloc_outputs(torch.from_numpy(w).cuda(), pack_int4=True, dequant=True, dequant_bf16=True) for w in ws2]
+    scs = [None, _clip_scales(ws2[1], 4, seed=1), _clip_scales(ws2[2], 4, seed=2)]
+    for b, sc in zip(bufs, scs):
+        b.codes.fill_(-128)
+        if sc is not None:
+            b.scales_in = torch.from_numpy(sc).cuda()
+    sq.squant_quantize_model(bufs, bits=4, flags=flags)
+    sq.squant_device_status()
+    for b, w, sc in zip(bufs, ws2, scs):
+        r = oracle.quantize_layer(w, bits=4, flags=flags, details=True, scales_in=sc)
+        assert np.array_equal(b.codes.cpu().numpy(), r.codes), w.shape
+        assert np.array_equal(b.kernel_err.cpu().numpy().view(np.uint32), r.kernel_err.view(np.uint32)), w.shape
+        assert np.array_equal(b.channel_err.cpu().numpy().view(np.uint32), r.channel_err.view(np.uint32))
+        assert np.array_equal(b.dequant.cpu().numpy().view(np.uint32), r.dequant.view(np.uint32))
+        assert np.array_equal(b.dequant_bf16.view(torch.int16).cpu().numpy().view(np.uint16), r.dequant_bf16)
+    with pytest.raises(sq.SquantError):   # beyond the select key's 18 index bits
+        sq.squant_plan_info([(1, 262144, 1, 1)])
