@@ -103,7 +103,7 @@ int validate(const squant_layer *layers, int32_t n_layers, const squant_options 
 
 // Device-side descriptor of one layer: group size and the layout of a group's shared-memory
 // slice.  Returns the dynamic shared memory one CTA needs for this layer.
-int64_t layout_layer(const squant_layer &l, LayerDesc &d, unsigned mode)
+int64_t layout_layer(const squant_layer &l, LayerDesc &d, unsigned mode, unsigned flags)
 {
     d.w = l.w; d.codes = l.codes; d.scales = l.scales; d.kerr = l.kernel_err; d.cerr = l.channel_err; d.deq = l.dequant;
     d.sin = l.scales_in; d.deq16 = l.dequant_bf16;
@@ -111,6 +111,16 @@ int64_t layout_layer(const squant_layer &l, LayerDesc &d, unsigned mode)
     d.g = group_size(d.NK);
     d.g_shift = 0;
     while ((1 << d.g_shift) < d.g) ++d.g_shift;
+    // Depthwise layers (one kernel per output channel) with plain outputs: a whole channel per thread.
+    // SQuant-C is void there once SQuant-K has run; without K (E|C) the channel step is real.
+    if (d.N == 1 && d.K <= 64 && !l.scales_in && !l.dequant && !l.dequant_bf16 && !(flags & SQUANT_FLAG_PACK_INT4) &&
+        ((mode & SQUANT_MODE_K) || !(mode & SQUANT_MODE_C))) {
+        d.g = 1;
+        d.g_shift = 0;
+        d.off_codes = 4 * d.K; d.off_ev = 0; d.off_vv = 0; d.off_vi = 0; d.off_hist = 0; d.off_red = 0;
+        d.slice_bytes = align16(5 * d.K);
+        return static_cast<int64_t>(sq::kCtaThreads) * d.slice_bytes;
+    }
     int off = align16(4 * d.NK);              // staged weights
     d.off_codes = off; off += align16(d.NK);  // staged codes
     const bool ec_only = (mode & SQUANT_MODE_C) && !(mode & SQUANT_MODE_K);   // elements are the candidates
@@ -140,7 +150,7 @@ int build_plan(const squant_layer *layers, int32_t n_layers, const squant_option
     std::vector<Batch> batches;
     for (int i = 0; i < n_layers; ++i) {
         LayerDesc &d = p.layers[i];
-        const int64_t cta_smem = layout_layer(layers[i], d, o.mode);
+        const int64_t cta_smem = layout_layer(layers[i], d, o.mode, o.flags);
         const int groups = sq::kCtaThreads / d.g;
         if (cta_smem > max_smem) return SQUANT_ERR_TOO_WIDE;
         if (cta_smem > p.smem_bytes) p.smem_bytes = static_cast<int>(cta_smem);
@@ -197,7 +207,7 @@ int build_param_plan(const squant_layer *layers, int32_t n_layers, const squant_
     std::vector<LayerDesc> descs(n_layers);
     std::vector<int> order, piped;
     for (int i = 0; i < n_layers; ++i) {
-        const int64_t cta_smem = layout_layer(layers[i], descs[i], o.mode);
+        const int64_t cta_smem = layout_layer(layers[i], descs[i], o.mode, o.flags);
         if (cta_smem > max_smem || descs[i].NK > kMaxChannelElems) {
             // a cluster of 2, 4 or 8 CTAs per output channel, each with an even number of kernels
             if ((o.mode & SQUANT_MODE_C) && !(o.mode & SQUANT_MODE_K) && descs[i].K > 1) return SQUANT_ERR_TOO_WIDE;   // E|C selects among elements: one CTA only

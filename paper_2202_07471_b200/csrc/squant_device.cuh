@@ -781,6 +781,100 @@ __device__ __forceinline__ void emit_channel(const LayerDesc &L, int m, const Gr
     }
 }
 
+// ---------------------------------------------------------------- one kernel by a whole warp
+// The same as kernel_generic for a channel with few kernels of many elements (a 7x7 stem has three
+// per output channel): thread-per-kernel would leave 29 lanes idle while three walk up to 25
+// arg-max rounds over 49 keys each.  Here the warp takes one kernel at a time, lane l holding
+// elements l, l + 32, ...: every round is a lane-local scan and three warp reductions (largest
+// key, lowest index among its holders).  Called by all 32 lanes; the results are warp-uniform.
+__device__ __forceinline__ void kernel_warp(float *wk, int K, float s, bool do_k, int8_t *ck, int lane,
+                                            long long &e_out, int &v_out, int &idx_out)
+{
+    int *Pk = reinterpret_cast<int *>(wk);
+    long long e = 0;
+    for (int i = lane; i < K; i += 32) {
+        int q, P;
+        squant_e(wk[i], s, q, P);
+        ck[i] = static_cast<int8_t>(q);
+        Pk[i] = P;
+        e += P;
+    }
+    {   // |e| <= K / 2 < 2^15 units: hi and lo halves cannot overflow 32 bits over a warp
+        const int hi = __reduce_add_sync(kFull, static_cast<int>(e >> 16));
+        const int lo = __reduce_add_sync(kFull, static_cast<int>(e & 0xffff));
+        e = (static_cast<long long>(hi) << 16) + lo;
+    }
+    __syncwarp();
+    int v = 0, idx = 0;
+    if (e != 0) {
+        const int sgn = e > 0 ? 1 : -1;
+        const long long abs_e = e > 0 ? e : -e;
+        const int k = do_k ? flip_count(abs_e) : 0;
+        int flips = 0, last = -1, cand = -1;
+        for (int r = 0; r <= k; ++r) {
+            int best = 0, bi = 0x7fffffff;
+            for (int i = lane; i < K; i += 32) {
+                const int key = sgn * Pk[i];
+                if (key > best) { best = key; bi = i; }   // strict: the lane's lowest index wins its ties
+            }
+            const int top = __reduce_max_sync(kFull, best);
+            if (top <= 0) break;
+            const int who = __reduce_min_sync(kFull, best == top ? bi : 0x7fffffff);
+            if (r < k) {
+                if (who % 32 == lane) {
+                    Pk[who] -= sgn * kOne;
+                    ck[who] = static_cast<int8_t>(ck[who] - sgn);
+                }
+                __syncwarp();
+                last = who;
+                ++flips;
+            } else {
+                cand = who;
+            }
+        }
+        e -= static_cast<long long>(sgn) * flips * kOne;
+        if (static_cast<long long>(flips) * kOne > abs_e) {   // Over SQuant: flip back candidate
+            idx = last;
+            v = Pk[last];
+        } else if (cand >= 0) {                               // Under SQuant: next un-flipped
+            idx = cand;
+            v = Pk[cand];
+        }
+    }
+    e_out = e;
+    v_out = v;
+    idx_out = idx;
+}
+
+// ---------------------------------------------------------------- one whole channel per thread
+// Depthwise convolutions: one kernel per output channel (N = 1), so SQuant-C has nothing to do once
+// SQuant-K has run (the channel's sum is the kernel's, within one half), and a channel is a handful
+// of weights.  One thread takes the whole channel - absmax, scale, SQuant-E/K, stores - and a
+// 256-thread CTA takes 256 channels instead of eight.  slice: K floats and K code bytes of the thread.
+__device__ __forceinline__ void channel_single(const LayerDesc &L, int m, unsigned char *slice, int qmax, unsigned mode)
+{
+    const int K = L.K;
+    float *wk = reinterpret_cast<float *>(slice);
+    int8_t *ck = reinterpret_cast<int8_t *>(slice + 4 * K);
+    const float *wg = L.w + static_cast<size_t>(m) * K;
+    float amax = 0.0f;
+    for (int i = 0; i < K; ++i) {
+        const float t = __ldcs(wg + i);
+        wk[i] = t;
+        amax = fmaxf(amax, fabsf(t));
+    }
+    const float s = (amax < 0x1p-100f) ? 1.0f : __fdiv_rn(amax, static_cast<float>(qmax));
+    long long e;
+    int v, idx;
+    kernel_generic(wk, K, s, (mode & 2u) != 0, ck, e, v, idx);
+    int8_t *cg = L.codes + static_cast<size_t>(m) * K;
+    for (int i = 0; i < K; ++i) cg[i] = ck[i];
+    const float ef = __fmul_rn(__ll2float_rn(e), 0x1p-30f);
+    L.scales[m] = s;
+    if (L.kerr) L.kerr[m] = ef;
+    if (L.cerr) L.cerr[m] = ef;
+}
+
 // ---------------------------------------------------------------- channel body, any kernel size
 template <int KT>
 __device__ __forceinline__ void channel_body(const LayerDesc &L, int m, const Group &G,
@@ -801,6 +895,25 @@ __device__ __forceinline__ void channel_body(const LayerDesc &L, int m, const Gr
     const bool keep = do_k || KT == 1 || K == 1;
     float *kerr = L.kerr ? L.kerr + static_cast<size_t>(m) * N : nullptr;
     long long esum = 0;
+    if (KT == 0 && K >= 16 && 4 * N <= G.g) {
+        // few kernels of many elements: a warp per kernel, lanes over its elements
+        const int lane = G.t & 31;
+        for (int n = G.t >> 5; n < N; n += G.g >> 5) {
+            long long e1;
+            int v, idx;
+            kernel_warp(wbuf + static_cast<size_t>(n) * K, K, s, do_k, cbuf + static_cast<size_t>(n) * K, lane, e1, v, idx);
+            if (lane == 0) {
+                if (keep) {
+                    ev[n] = static_cast<int>(e1);
+                    vv[n] = v;
+                    vi[n] = static_cast<unsigned short>(idx);
+                } else if (kerr) {
+                    kerr[n] = __fmul_rn(__ll2float_rn(e1), 0x1p-30f);
+                }
+                esum += e1;
+            }
+        }
+    } else
     for (int n = G.t; n < N; n += G.g) {
         long long e1;
         if (KT == 1) {
@@ -1426,6 +1539,11 @@ __global__ void debug_wait_kernel(int max_polls)
 __device__ __forceinline__ void run_item(const LayerDesc &L, int ch0, unsigned char *smem, int qmax,
                                          unsigned mode)
 {
+    if (L.g == 1) {   // depthwise: one channel per thread
+        const int m1 = ch0 + static_cast<int>(threadIdx.x);
+        if (m1 < L.M) channel_single(L, m1, smem + static_cast<size_t>(threadIdx.x) * L.slice_bytes, qmax, mode);
+        return;
+    }
     Group G;
     G.g = L.g;
     G.t = threadIdx.x & (L.g - 1);

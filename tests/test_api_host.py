@@ -43,7 +43,8 @@ def test_plan_geometry_for_the_five_configs():
     assert _info(W.WORKLOADS["large_layer"].shapes)["grid_ctas"] == 8 * 2048
     # small channels share a CTA: 8 warps, one channel each
     assert _info([(64, 64, 3, 3)])["grid_ctas"] == 8   # 64 channels, 8 one-warp groups per 256-thread block
-    assert _info([(33, 1, 3, 3)])["grid_ctas"] == 5
+    assert _info([(33, 7, 3, 3)])["grid_ctas"] == 5
+    assert _info([(600, 1, 3, 3)])["grid_ctas"] == 3   # depthwise: a whole channel per thread, 256 per block
 
 
 @pytest.mark.parametrize("shape,kw,code", [
