@@ -236,6 +236,16 @@ int squant_device_status(void);
  * next squant_device_status returns SQUANT_ERR_TIMEOUT and the context stays usable.
  */
 int squant_debug_set_status(int value);
+/*
+ * The checked build of the library (libsquant_debug.so, compiled with -DSQUANT_DEBUG_BOUNDS; the
+ * stand-in for a memory checker on small test cases): its kernels verify every index they form
+ * into shared memory and into the launch table, and take each 3x3 channel's error sum a second
+ * time from its final codes by plain division.  This call waits for the device, returns the number
+ * of failed checks since the last call and the site number of the first (both 0 when all is well)
+ * and clears them.  Return value: 1 if the library was built with the checks, 0 if not (the
+ * counters then stay 0), or a negative error.
+ */
+int squant_debug_violations(int32_t *count, int32_t *first_site);
 int squant_debug_wait_expires(int32_t max_polls, void *cuda_stream);
 
 /* Number of kernels this library has launched in this process (all entry points). */

@@ -24,7 +24,7 @@ NOALLOC_MAX_CTAS = 32768
 
 EXPORTS = ("squant_quantize_layer", "squant_quantize_layer_noalloc", "squant_quantize_model", "squant_quantize_model_host",
            "squant_plan_info", "squant_selfcheck_division", "squant_device_status", "squant_launch_count", "squant_strerror", "squant_last_cuda_error",
-           "squant_shutdown", "squant_debug_set_status", "squant_debug_wait_expires")
+           "squant_shutdown", "squant_debug_set_status", "squant_debug_wait_expires", "squant_debug_violations")
 
 
 class SquantError(RuntimeError):
@@ -68,6 +68,8 @@ def load_library() -> ctypes.CDLL:
     for f in ("squant_quantize_layer", "squant_quantize_layer_noalloc", "squant_quantize_model", "squant_quantize_model_host",
               "squant_plan_info", "squant_selfcheck_division", "squant_device_status", "squant_shutdown"):
         getattr(lib, f).restype = ctypes.c_int
+    lib.squant_debug_violations.argtypes = [i32p, i32p]
+    lib.squant_debug_violations.restype = ctypes.c_int
     lib.squant_debug_set_status.argtypes = [ctypes.c_int]
     lib.squant_debug_set_status.restype = ctypes.c_int
     lib.squant_debug_wait_expires.argtypes = [ctypes.c_int32, vp]
@@ -244,6 +246,22 @@ def squant_selfcheck_division(scales, bits: int = 4):
 def squant_device_status() -> None:
     """Synchronise the current device; raise SquantError(-10) if a kernel gave up a bounded wait."""
     _check(load_library().squant_device_status())
+
+
+def use_library(path: Optional[str]) -> None:
+    """Switch to another build of the library (the checked one, for tests); None: the regular one."""
+    global _lib, LIB_PATH
+    _lib = None
+    LIB_PATH = path if path is not None else os.path.join(_HERE, "libsquant.so")
+
+
+def squant_debug_violations():
+    """(checked build?, failed checks since the last call, site of the first)."""
+    n, site = ctypes.c_int32(), ctypes.c_int32()
+    rc = load_library().squant_debug_violations(ctypes.byref(n), ctypes.byref(site))
+    if rc < 0:
+        _check(rc)
+    return bool(rc), n.value, site.value
 
 
 def squant_debug_set_status(value: int) -> None:

@@ -10,6 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsquant.so")
+LIB_DEBUG = os.path.join(HERE, "libsquant_debug.so")   # the checked build (-DSQUANT_DEBUG_BOUNDS), for tests on small cases
 SOURCES = [os.path.join(CSRC, "squant.cu")]
 DEPS = SOURCES + sorted(glob.glob(os.path.join(CSRC, "*.cuh"))) + [os.path.join(ROOT, "include", "squant.h")]
 
@@ -27,21 +28,23 @@ def nvcc_path() -> str:
     return p
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and os.path.exists(LIB) and all(
-            os.path.getmtime(LIB) >= os.path.getmtime(d) for d in DEPS):
-        return LIB
-    tmp = LIB + f".tmp{os.getpid()}"
-    cmd = [nvcc_path(), *NVCC_FLAGS, "-o", tmp, *SOURCES]
+def build(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
+    lib = LIB_DEBUG if debug else LIB
+    if not force and os.path.exists(lib) and all(
+            os.path.getmtime(lib) >= os.path.getmtime(d) for d in DEPS):
+        return lib
+    tmp = lib + f".tmp{os.getpid()}"
+    cmd = [nvcc_path(), *NVCC_FLAGS, *(["-DSQUANT_DEBUG_BOUNDS"] if debug else []), "-o", tmp, *SOURCES]
     res = subprocess.run(cmd, capture_output=True, text=True)
     if verbose or res.returncode != 0:
         print(res.stdout)
         print(res.stderr)
     if res.returncode != 0:
-        raise RuntimeError("nvcc failed building libsquant.so")
-    os.replace(tmp, LIB)
-    return LIB
+        raise RuntimeError("nvcc failed building " + os.path.basename(lib))
+    os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":
     print(build(force=True, verbose=True))
+    print(build(force=True, debug=True))

@@ -720,6 +720,26 @@ int squant_device_status(void)
     return SQUANT_ERR_TIMEOUT;
 }
 
+int squant_debug_violations(int32_t *count, int32_t *first_site)
+{
+    std::lock_guard<std::mutex> lock(g_mutex);
+    SQ_CUDA(cudaDeviceSynchronize());
+    unsigned n = 0;
+    int site = 0;
+    SQ_CUDA(cudaMemcpyFromSymbol(&n, sq::g_debug_violations, sizeof(n)));
+    SQ_CUDA(cudaMemcpyFromSymbol(&site, sq::g_debug_site, sizeof(site)));
+    if (count) *count = static_cast<int32_t>(n);
+    if (first_site) *first_site = site;
+    const unsigned zero = 0;
+    SQ_CUDA(cudaMemcpyToSymbol(sq::g_debug_violations, &zero, sizeof(zero)));
+    SQ_CUDA(cudaMemcpyToSymbol(sq::g_debug_site, &zero, sizeof(int)));
+#ifdef SQUANT_DEBUG_BOUNDS
+    return 1;   // this library was built with the checks
+#else
+    return SQUANT_OK;
+#endif
+}
+
 int squant_debug_set_status(int value)
 {
     std::lock_guard<std::mutex> lock(g_mutex);

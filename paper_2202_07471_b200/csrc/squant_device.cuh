@@ -68,6 +68,34 @@ struct Group {
     }
 };
 
+// ---------------------------------------------------------------- checked build
+// Built with -DSQUANT_DEBUG_BOUNDS (a second library, for tests on small cases), the kernels check
+// the indices they form into shared memory and into the launch table against their bounds, and
+// recompute every channel's error sum from its final codes and staged weights; a failed check is
+// counted and its site recorded, the access it guards is skipped where it can be.  The regular
+// build compiles the checks away.
+__device__ unsigned g_debug_violations = 0;
+__device__ int g_debug_site = 0;
+#ifdef SQUANT_DEBUG_BOUNDS
+__device__ __noinline__ void sq_debug_fail(int site)
+{
+    atomicAdd(&g_debug_violations, 1u);
+    atomicCAS(&g_debug_site, 0, site);
+}
+#define SQ_DBG(cond, site) do { if (!(cond)) sq_debug_fail(site); } while (0)
+#define SQ_DBG_OK(cond, site) ((cond) ? true : (sq_debug_fail(site), false))
+#else
+#define SQ_DBG(cond, site) ((void)0)
+#define SQ_DBG_OK(cond, site) (true)
+#endif
+
+__device__ __forceinline__ unsigned dynamic_smem_bytes()
+{
+    unsigned v;
+    asm("mov.u32 %0, %%dynamic_smem_size;" : "=r"(v));
+    return v;
+}
+
 // ---------------------------------------------------------------- bulk async copies (TMA)
 // Set to a non-zero code by a kernel whose bounded wait on a bulk copy ran out; read and cleared
 // by squant_device_status().
@@ -575,6 +603,7 @@ __device__ __forceinline__ bool kernel9_select(const float (&Psf)[9], float ef, 
     // Every key carries the index of a real element, so the positions below are 0..8 whatever
     // the input; ranks 1 and 2 are read-modify-written unconditionally (a zero change when the
     // flip does not apply), ranks 3 and 4 are rare enough for a branch.
+    SQ_DBG((~m1 & 15) < 9 && (~m2 & 15) < 9 && (~m3 & 15) < 9 && (~m4 & 15) < 9, 1);   // every key carries a real element's index
     {
         unsigned char *p1 = cb + (~m1 & 15);
         *p1 = static_cast<unsigned char>(*p1 - ((ok & (jx >= 1u)) ? sgn : 0));
@@ -952,13 +981,24 @@ __device__ __forceinline__ void channel_body(const LayerDesc &L, int m, const Gr
                 if (ck != 0 && ck >= T) {
                     e1 -= sgn_c * kOne;
                     const size_t j = (KT == 1) ? n : static_cast<size_t>(n) * K + vi[n];
-                    cbuf[j] = static_cast<int8_t>(cbuf[j] - sgn_c);
+                    if (SQ_DBG_OK(j < static_cast<size_t>(L.NK) && (KT == 1 || vi[n] < K), 2)) cbuf[j] = static_cast<int8_t>(cbuf[j] - sgn_c);
                 }
             }
             if (kerr) kerr[n] = __fmul_rn(__int2float_rn(e1), 0x1p-30f);
         }
     }
     G.sync();
+#ifdef SQUANT_DEBUG_BOUNDS
+    // Checked build, kernels kept in shared memory: the perturbations staged after SQuant-K, summed
+    // again, minus one unit per channel flip must equal the channel sum.
+    if (KT == 0 && ((mode & 4u) || L.cerr)) {
+        const int *Pall = reinterpret_cast<const int *>(slice);
+        long long chk = 0;
+        for (int j = G.t; j < N * K; j += G.g) chk += Pall[j];
+        chk = group_sum(G, chk, slice + L.off_red);
+        if (G.t == 0) SQ_DBG(chk - static_cast<long long>(sgn_c) * k_eff * kOne == ec, 9);
+    }
+#endif
 
     // ---- codes, scale, channel error (the staged weights / perturbations are dead: scratch)
     emit_channel(L, m, G, reinterpret_cast<const unsigned char *>(cbuf), slice, s, ec, mode);
@@ -1275,6 +1315,7 @@ __device__ __forceinline__ void finish_channel_hist(const LayerDesc &L, int m, c
                         }
                     }
                     if (take) {
+                        SQ_DBG(n < N && (KT == 1 || vi[n] < 9), 3);
                         unsigned char *bp = cbuf + (KT == 1 ? n : n * 9 + vi[n]);
                         *bp = static_cast<unsigned char>(*bp - sgn_c);
                         if (kerr) kerr[n] = __fmul_rn(__int2float_rn(ev[n] - sgn_c * kOne), 0x1p-30f);
@@ -1293,6 +1334,7 @@ __device__ __forceinline__ void finish_channel_hist(const LayerDesc &L, int m, c
                 rank += (o.x > me.x || (o.x == me.x && o.y < me.y)) ? 1 : 0;
             }
             if (rank < rem) {
+                SQ_DBG(me.y >= 0 && me.y < N && cb <= kListCap, 4);
                 unsigned char *bp = cbuf + (KT == 1 ? me.y : me.y * 9 + vi[me.y]);
                 *bp = static_cast<unsigned char>(*bp - sgn_c);
                 if (kerr) kerr[me.y] = __fmul_rn(__int2float_rn(ev[me.y] - sgn_c * kOne), 0x1p-30f);
@@ -1301,6 +1343,24 @@ __device__ __forceinline__ void finish_channel_hist(const LayerDesc &L, int m, c
         G.sync();
     }
 
+#ifdef SQUANT_DEBUG_BOUNDS
+    // Checked build, grouped kernel, 3x3: the staged weights are still there, so the channel's error
+    // sum can be taken again from scratch - plain IEEE division of every weight, perturbation of
+    // its FINAL code - and must equal what the selection machinery arrived at.
+    if (KT == 9 && w_release == nullptr && pack_scratch == nullptr) {
+        G.sync();
+        const float *wchk = reinterpret_cast<const float *>(slice);
+        long long chk = 0;
+        for (int j = G.t; j < 9 * N; j += G.g) {
+            // rounded code and its perturbation (that difference is exact), then whole steps for the flips
+            const float x = __fdiv_rn(wchk[j], s), q0 = rintf(x);
+            const long long P0 = __float2ll_rn(__fmul_rn(__fsub_rn(q0, x), 1073741824.0f));
+            chk += P0 + (static_cast<long long>(static_cast<signed char>(cbuf[j])) - __float2int_rn(q0)) * kOne;
+        }
+        chk = group_sum(G, chk, red);
+        if (G.t == 0) SQ_DBG(chk == ec, 8);
+    }
+#endif
     // ---- codes, scale, channel error (the staged weights / perturbations are dead: scratch)
     emit_channel(L, m, G, cbuf, pack_scratch ? pack_scratch : slice, s, ec, mode);
 }
@@ -1552,6 +1612,9 @@ __device__ __forceinline__ void run_item(const LayerDesc &L, int ch0, unsigned c
     const int m = ch0 + gi;
     if (m >= L.M) return;   // the whole group leaves together; it shares no barrier with others
     unsigned char *slice = smem + static_cast<size_t>(gi) * L.slice_bytes;
+    SQ_DBG(ch0 >= 0 && L.g >= 32 && (L.g & (L.g - 1)) == 0 && (1 << L.g_shift) == L.g, 5);
+    SQ_DBG(static_cast<size_t>(gi + 1) * L.slice_bytes <= dynamic_smem_bytes(), 6);
+    SQ_DBG(L.off_red + 256 <= L.slice_bytes && L.off_hist + 4 * kHistBins <= L.off_red && L.off_codes + L.NK <= L.slice_bytes, 7);
     const float s = stage_channel(L, m, G, slice, qmax);
     if (s == 0.0f) return;   // staging wait ran out (status word set); nothing is written
     if (L.sin) {   // Algorithm 1 with its scale as an input

@@ -563,3 +563,32 @@ def test_channels_wider_than_one_thread_block():
         assert np.array_equal(b.dequant_bf16.view(torch.int16).cpu().numpy().view(np.uint16), r.dequant_bf16)
     with pytest.raises(sq.SquantError):   # beyond the select key's 18 index bits
         sq.squant_plan_info([(1, 262144, 1, 1)])
+
+
+def test_checked_build_finds_no_violation_on_small_cases():
+    """The checked build of the library (every shared-memory / table index verified, each 3x3
+    channel's error sum taken a second time from its final codes by plain division) runs the
+    sweep of small shapes, the 3x3 cases the fast selection hands back, and a cluster case:
+    no check fails, and its results are the regular build's."""
+    from paper_2202_07471_b200 import build as lib_build
+    import os
+    if not os.path.exists(lib_build.LIB_DEBUG):
+        pytest.skip("libsquant_debug.so has not been built")
+    ws = [adversarial_layer(s, seed=9 + i) for i, s in enumerate(SWEEP_SHAPES)] + [redo_layer(64, 4, seed=4), redo_layer(2048, 4)]
+    ref = run_gpu(ws, 4, EKC)
+    sq.use_library(lib_build.LIB_DEBUG)
+    try:
+        checked, n, site = sq.squant_debug_violations()
+        assert checked and n == 0
+        for mode in (EKC, EK, sq.MODE_E | sq.MODE_C):
+            bufs = run_gpu(ws, 4, mode)
+            _, n, site = sq.squant_debug_violations()
+            assert n == 0, f"{n} failed checks, first at site {site}, mode {mode}"
+            if mode == EKC:
+                for a, b in zip(bufs, ref):
+                    assert torch.equal(a.codes, b.codes) and torch.equal(a.kernel_err.view(torch.int32), b.kernel_err.view(torch.int32))
+        (b,) = run_gpu([W.random_layer((2, 70001, 1, 1), seed=2)], 4, EKC)
+        assert sq.squant_debug_violations()[1] == 0
+    finally:
+        sq.use_library(None)
+    assert sq.squant_debug_violations()[0] is False      # the regular build has no checks
