@@ -378,7 +378,7 @@ def run_cuda(args):
     roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
             "frac": achieved / peak, "traffic": traffic, "peak_kind": f"of {peak_kind}",
             "peak_ncu": nominal, "frac_of_ncu_peak": achieved / nominal,
-            "kernel": "squant_pipe_kernel", "kernel_ms": kernel_ms, "algorithmic_bytes_per_launch": alg}
+            "kernel": "squant_stream_kernel", "kernel_ms": kernel_ms, "algorithmic_bytes_per_launch": alg}
     if traffic:   # what actually crossed the DRAM interface (part of the output is still in L2 at kernel end)
         roof["achieved_dram"] = traffic / (kernel_ms * 1e-3) / 1e9
         roof["frac_dram_of_measured"] = roof["achieved_dram"] / peak

@@ -14,6 +14,7 @@
 
 #include "squant_device.cuh"
 #include "squant_pipe.cuh"
+#include "squant_stream.cuh"
 #include "squant_wide.cuh"
 
 namespace {
@@ -181,6 +182,21 @@ struct ParamPlan {
     // pipelined kernel (layers of long 3x3 channels): one item per output channel
     std::vector<sq::LaunchTable> pipe_tables;
     std::vector<int> pipe_items, pipe_set_stride, pipe_slot;
+    std::vector<int> pipe_stream;   // 1: the launch goes to the streaming kernel (plain int8 output); pipe_set_stride then
+    std::vector<int> pipe_nmax;     // holds the longest channel in weights and pipe_nmax the same in kernels
+    // Scratch of the streaming kernel's launches (what SQuant-C needs of every kernel one step later: two
+    // sets of 18 KB per thread block), allocated at the plan's first launch, freed with the plan.
+    mutable std::vector<void *> pipe_scratch;
+    ParamPlan() = default;
+    ParamPlan(ParamPlan &&) = default;
+    ParamPlan &operator=(ParamPlan &&) = default;
+    ParamPlan(const ParamPlan &) = delete;
+    ParamPlan &operator=(const ParamPlan &) = delete;
+    ~ParamPlan()
+    {
+        for (void *q : pipe_scratch)
+            if (q) cudaFree(q);
+    }
     mutable bool slots_clean = false;   // the work counters of pipe_slot have been zeroed on the stream of the plan's first launch
 };
 
@@ -197,6 +213,14 @@ bool pipe_eligible(const squant_layer &l, const LayerDesc &d, const squant_optio
     return 2 * d.slice_bytes + sq::kPipeCtrlBytes <= max_smem;
 }
 
+// Of those, the streaming kernel takes the layers with plain int8 codes and nothing else to emit.
+bool stream_eligible(const squant_layer &l, const LayerDesc &d, const squant_options &o, int max_smem)
+{
+    if (l.dequant || l.dequant_bf16 || (o.flags & SQUANT_FLAG_PACK_INT4)) return false;
+    if (d.N > 4 * sq::kStreamQuantThreads) return false;   // one quad of kernels per quantizer thread
+    return sq::stream_layout(d.NK, d.N).total <= max_smem;
+}
+
 int build_param_plan(const squant_layer *layers, int32_t n_layers, const squant_options &o,
                      int max_smem, ParamPlan &p)
 {
@@ -205,7 +229,7 @@ int build_param_plan(const squant_layer *layers, int32_t n_layers, const squant_
              ((o.flags & SQUANT_FLAG_NARROW_RANGE) ? 0u : sq::kModeWideRange);
     p.smem_bytes = 0;
     std::vector<LayerDesc> descs(n_layers);
-    std::vector<int> order, piped;
+    std::vector<int> order, piped, streamed;
     for (int i = 0; i < n_layers; ++i) {
         const int64_t cta_smem = layout_layer(layers[i], descs[i], o.mode, o.flags);
         if (cta_smem > max_smem || descs[i].NK > kMaxChannelElems) {
@@ -222,14 +246,16 @@ int build_param_plan(const squant_layer *layers, int32_t n_layers, const squant_
             continue;
         }
         if (pipe_eligible(layers[i], descs[i], o, max_smem)) {
-            piped.push_back(i);
+            (stream_eligible(layers[i], descs[i], o, max_smem) ? streamed : piped).push_back(i);
             continue;
         }
         if (cta_smem > p.smem_bytes) p.smem_bytes = static_cast<int>(cta_smem);
         order.push_back(i);
     }
-    for (size_t base = 0; base < piped.size(); base += sq::kMaxParamLayers) {
-        const int n = static_cast<int>(std::min<size_t>(piped.size() - base, sq::kMaxParamLayers));
+    for (int kind = 0; kind < 2; ++kind) {
+    const std::vector<int> &piped_k = kind ? streamed : piped;
+    for (size_t base = 0; base < piped_k.size(); base += sq::kMaxParamLayers) {
+        const int n = static_cast<int>(std::min<size_t>(piped_k.size() - base, sq::kMaxParamLayers));
         p.pipe_tables.emplace_back();
         sq::LaunchTable &t = p.pipe_tables.back();
         std::memset(&t, 0, sizeof(t));
@@ -237,7 +263,7 @@ int build_param_plan(const squant_layer *layers, int32_t n_layers, const squant_
         for (int st = 1; st < n; st <<= 1) t.top_step = st;
         int items = 0, stride = 0;
         for (int j = 0; j < n; ++j) {
-            const LayerDesc &d = descs[piped[base + j]];
+            const LayerDesc &d = descs[piped_k[base + j]];
             t.layers[j] = d;
             t.first_item[j] = items;
             items += d.M;
@@ -257,10 +283,19 @@ int build_param_plan(const squant_layer *layers, int32_t n_layers, const squant_
             d.off_codes = wd.off_codes; d.off_ev = wd.off_ev; d.off_vv = wd.off_vv; d.off_vi = wd.off_vi;
             d.off_hist = wd.off_hist; d.off_red = wd.off_red; d.slice_bytes = wd.slice_bytes;
         }
+        int nk_max = 0, n_max = 0;
+        for (int j = 0; j < n; ++j) {
+            nk_max = std::max(nk_max, t.layers[j].NK);
+            n_max = std::max(n_max, t.layers[j].N);
+        }
         p.pipe_items.push_back(items);
-        p.pipe_set_stride.push_back(stride);
+        p.pipe_set_stride.push_back(kind ? nk_max : stride);
+        p.pipe_stream.push_back(kind);
+        p.pipe_scratch.push_back(nullptr);
+        p.pipe_nmax.push_back(n_max);
         p.pipe_slot.push_back(g_next_slot);
         g_next_slot = (g_next_slot + 1) % sq::kTicketSlots;
+    }
     }
     n_layers = static_cast<int32_t>(order.size());   // the grouped kernel takes the rest
     // Estimated duration of one CTA of the layer.  Kernel sizes other than 1x1 and 3x3 take the
@@ -329,6 +364,8 @@ int device_smem_limit(int device, int &limit)
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, v));
         SQ_CUDA(cudaFuncSetAttribute(sq::squant_wide_kernel,
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, v));
+        SQ_CUDA(cudaFuncSetAttribute(sq::squant_stream_kernel,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, v));
         int sms = 0;
         SQ_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
         if (static_cast<int>(g_sm_count_by_device.size()) <= device) g_sm_count_by_device.resize(device + 1, 0);
@@ -396,9 +433,18 @@ int launch_plan(const ParamPlan &p, cudaStream_t stream)
         int device = 0;
         SQ_CUDA(cudaGetDevice(&device));
         const int grid = std::min(p.pipe_items[c], std::max(g_sm_count_by_device[device], 1));
-        const int smem = 2 * p.pipe_set_stride[c] + sq::kPipeCtrlBytes;
-        sq::squant_pipe_kernel<<<grid, sq::kPipeThreads, smem, stream>>>(p.pipe_tables[c], p.qmax, p.mode, p.pipe_items[c],
-                                                                     p.pipe_slot[c], p.pipe_set_stride[c]);
+        if (p.pipe_stream[c]) {
+            const int smem = sq::stream_layout(p.pipe_set_stride[c], p.pipe_nmax[c]).total;
+            if (!p.pipe_scratch[c])
+                SQ_CUDA(cudaMalloc(&p.pipe_scratch[c], static_cast<size_t>(std::max(g_sm_count_by_device[device], 1)) * 2 * sq::kStreamHeldBytes));
+            sq::squant_stream_kernel<<<grid, sq::kStreamThreads, smem, stream>>>(p.pipe_tables[c], p.qmax, p.mode, p.pipe_items[c],
+                                                                             p.pipe_slot[c], p.pipe_set_stride[c], p.pipe_nmax[c],
+                                                                             static_cast<unsigned char *>(p.pipe_scratch[c]));
+        } else {
+            const int smem = 2 * p.pipe_set_stride[c] + sq::kPipeCtrlBytes;
+            sq::squant_pipe_kernel<<<grid, sq::kPipeThreads, smem, stream>>>(p.pipe_tables[c], p.qmax, p.mode, p.pipe_items[c],
+                                                                         p.pipe_slot[c], p.pipe_set_stride[c]);
+        }
         SQ_CUDA(cudaGetLastError());
         g_launches.fetch_add(1, std::memory_order_relaxed);
     }
