@@ -184,7 +184,7 @@ struct ParamPlan {
     std::vector<int> pipe_items, pipe_set_stride, pipe_slot;
     std::vector<int> pipe_stream;   // 1: the launch goes to the streaming kernel (plain int8 output); pipe_set_stride then
     std::vector<int> pipe_nmax;     // holds the longest channel in weights and pipe_nmax the same in kernels
-    // Scratch of the streaming kernel's launches (what SQuant-C needs of every kernel one step later: two
+    // Scratch of the streaming kernel's launches (what SQuant-C needs of every kernel one step later: four
     // sets of 18 KB per thread block), allocated at the plan's first launch, freed with the plan.
     mutable std::vector<void *> pipe_scratch;
     ParamPlan() = default;
@@ -436,7 +436,7 @@ int launch_plan(const ParamPlan &p, cudaStream_t stream)
         if (p.pipe_stream[c]) {
             const int smem = sq::stream_layout(p.pipe_set_stride[c], p.pipe_nmax[c]).total;
             if (!p.pipe_scratch[c])
-                SQ_CUDA(cudaMalloc(&p.pipe_scratch[c], static_cast<size_t>(std::max(g_sm_count_by_device[device], 1)) * 2 * sq::kStreamHeldBytes));
+                SQ_CUDA(cudaMalloc(&p.pipe_scratch[c], static_cast<size_t>(std::max(g_sm_count_by_device[device], 1)) * sq::kStreamHeldSets * sq::kStreamHeldBytes));
             sq::squant_stream_kernel<<<grid, sq::kStreamThreads, smem, stream>>>(p.pipe_tables[c], p.qmax, p.mode, p.pipe_items[c],
                                                                              p.pipe_slot[c], p.pipe_set_stride[c], p.pipe_nmax[c],
                                                                              static_cast<unsigned char *>(p.pipe_scratch[c]));

@@ -50,7 +50,8 @@ constexpr int kStreamHelpThreads = 128;                     // channel warp, cop
                                                             // four warps, one per scheduler
 constexpr int kStreamThreads = kStreamHelpThreads + kStreamQuantThreads;
 constexpr int kStreamListCap = 128;                        // candidates ranked exactly inside the boundary bin
-constexpr int kStreamCtrlBytes = 2816;
+constexpr int kStreamQueueCap = 128;                       // quantizer threads per channel that hand their flips to the channel warp
+constexpr int kStreamCtrlBytes = 3328;
 
 // SQuant-C of one channel as the quantizers need it (sixteen bytes, read as one word).
 struct StreamDecision {
@@ -98,6 +99,8 @@ struct StreamCtrl {
     __align__(16) int4 fin[2];       // item (-1: end), layer, channel and scale bits of the step, handed on by the
                                      // quantizers to the channel warp
     int lcount[2];                   // entries in the boundary list
+    int qcount[2];                   // entries in the queue of concerned threads
+    unsigned short queue[2][kStreamQueueCap];   // quantizer threads with kernels to flip (or to rank)
     int abort;                       // a wait ran out: nobody waits any more
     unsigned amax[2];                // absmax of the staged channel (bit pattern), from the two scale warps
     int scratch[kStreamQuantWarps][12];                // nine words per quantizer warp for the exact routine
@@ -188,8 +191,10 @@ __device__ __noinline__ KernelOut kernel9_exact_smem(int *P, unsigned char *cb)
 // candidates, positions - waits in a scratch area in global memory (registers are what this kernel is
 // short of, and the flips are few: a dozen kernels in two thousand).  The thread itself keeps the
 // largest and the smallest candidate, which tell it whether any of its kernels is concerned at all.
-// Per CTA and buffer set: 512 x int4 sums, 512 x int4 candidates, 512 x 4 index bytes.
+// Per CTA and set: 512 x int4 sums, 512 x int4 candidates, 512 x 4 index bytes.
 constexpr int kStreamHeldBytes = kStreamQuantThreads * 36;   // one set
+constexpr int kStreamHeldSets = 4;   // by step modulo four, like the code buffers: a set is rewritten only after a wait
+                                     // that implies the channel warp is done with it
 struct StreamHeld {
     int vmax, vmin;   // largest and smallest of the four candidates (0 where there are no kernels)
     bool have;        // a previous channel exists
@@ -232,6 +237,51 @@ __device__ __forceinline__ void stream_rare(bool rare, const float2 (&P2)[18], f
             idx_out = static_cast<unsigned>(x.idx);
         }
         __syncwarp();
+    }
+}
+
+// SQuant-C's flips on the four kernels of quantizer thread t, whose details wait in the scratch set at
+// hset: kernels above the threshold are flipped here (code byte in the channel's staged codes, error sum
+// in global memory), members of the boundary bin go to the list for the exact ranking.
+__device__ __forceinline__ void stream_flip_thread(int t, const StreamDecision &D, unsigned long long T,
+                                                   const unsigned char *hset, unsigned char *codes, float *kerr_row,
+                                                   StreamListEntry *blist, int *lcount)
+{
+    // (written by another thread of this CTA two hand-overs ago: read past the L1)
+    const int4 he = __ldcg(reinterpret_cast<const int4 *>(hset) + t);
+    const int4 hv = __ldcg(reinterpret_cast<const int4 *>(hset + 16 * kStreamQuantThreads) + t);
+    const unsigned hidx = __ldcg(reinterpret_cast<const unsigned *>(hset + 32 * kStreamQuantThreads) + t);
+    const int hvv[4] = {hv.x, hv.y, hv.z, hv.w}, hee[4] = {he.x, he.y, he.z, he.w};
+    const int sgn_c = D.sgn_c;
+    const int t_min = D.kind == 2 ? 1 : min(D.t_all, D.t_list);
+#pragma unroll
+    for (int kq = 0; kq < 4; ++kq) {
+        const int a = hvv[kq] * sgn_c;
+        if (a >= t_min) {
+            const int n = 4 * t + kq;
+            const int pos = 36 * t + 9 * kq + min(static_cast<int>((hidx >> (8 * kq)) & 15u), 8);
+            bool take;
+            if (D.kind == 2) {
+                take = cand_key(hvv[kq], sgn_c, n) >= T;
+            } else {
+                take = a >= D.t_all;
+                if (!take) {
+                    const int at = atomicAdd(lcount, 1);
+                    if (at < kStreamListCap) {
+                        StreamListEntry en;
+                        en.a = a;
+                        en.n = n;
+                        en.pos = pos;
+                        en.e = hee[kq];
+                        blist[at] = en;
+                    }
+                }
+            }
+            if (take) {
+                codes[pos] = static_cast<unsigned char>(codes[pos] - sgn_c);
+                if (kerr_row) kerr_row[n] = __fmul_rn(__int2float_rn(hee[kq] - sgn_c * kOne), 0x1p-30f);
+            }
+        }
     }
 }
 
@@ -410,7 +460,7 @@ squant_stream_kernel(const __grid_constant__ LaunchTable tbl, int qmax, unsigned
         held.vmax = 0;
         held.vmin = 0;
         held.have = false;
-        unsigned char *hs = held_scratch + static_cast<size_t>(blockIdx.x) * (2 * kStreamHeldBytes);
+        unsigned char *hs = held_scratch + static_cast<size_t>(blockIdx.x) * (kStreamHeldSets * kStreamHeldBytes);
         auto held_e = [&](int set) { return reinterpret_cast<int4 *>(hs + set * kStreamHeldBytes) + qt; };
         auto held_v = [&](int set) { return reinterpret_cast<int4 *>(hs + set * kStreamHeldBytes + 16 * kStreamQuantThreads) + qt; };
         auto held_i = [&](int set) { return reinterpret_cast<unsigned *>(hs + set * kStreamHeldBytes + 32 * kStreamQuantThreads) + qt; };
@@ -427,7 +477,7 @@ squant_stream_kernel(const __grid_constant__ LaunchTable tbl, int qmax, unsigned
                 const unsigned long long prefix = ctrl->T[pb];
                 int *dh = reinterpret_cast<int *>(smem + lay.off_hist) + pb * kHistBins;
                 {
-                    const int4 hv = *held_v(pb);   // zeros where there are no kernels
+                    const int4 hv = *held_v(pj);   // zeros where there are no kernels
                     const int v[4] = {hv.x, hv.y, hv.z, hv.w};
 #pragma unroll
                     for (int kq = 0; kq < 4; ++kq) {
@@ -443,42 +493,16 @@ squant_stream_kernel(const __grid_constant__ LaunchTable tbl, int qmax, unsigned
             }
             const int t_min = D.kind == 2 ? 1 : min(D.t_all, D.t_list);
             if (D.kind != 0 && (D.sgn_c > 0 ? held.vmax : -held.vmin) >= t_min) {   // rare per thread (v = 0 where there are no kernels)
-                const int sgn_c = D.sgn_c;
-                const int4 hv = *held_v(pb), he = *held_e(pb);
-                const int hvv[4] = {hv.x, hv.y, hv.z, hv.w}, hee[4] = {he.x, he.y, he.z, he.w};
-                const unsigned hidx = *held_i(pb);
-                unsigned char *pcodes = smem + lay.off_codes + static_cast<size_t>(pj) * lay.c_bytes + qt * 36;
-                float *pkerr = ctrl->kprev[pj] ? ctrl->kprev[pj] + 4 * qt : nullptr;
-                StreamListEntry *blist = reinterpret_cast<StreamListEntry *>(smem + lay.off_list) + pb * kStreamListCap;
-#pragma unroll
-                for (int kq = 0; kq < 4; ++kq) {
-                    const int a = hvv[kq] * sgn_c;
-                    if (a >= t_min) {   // rare
-                        const int n = 4 * qt + kq;
-                        const int pos = 9 * kq + static_cast<int>((hidx >> (8 * kq)) & 15u);
-                        bool take;
-                        if (D.kind == 2) {
-                            take = cand_key(hvv[kq], sgn_c, n) >= ctrl->T[pb];
-                        } else {
-                            take = a >= D.t_all;
-                            if (!take) {
-                                const int at = atomicAdd(&ctrl->lcount[pb], 1);
-                                if (at < kStreamListCap) {
-                                    StreamListEntry en;
-                                    en.a = a;
-                                    en.n = n;
-                                    en.pos = 36 * qt + pos;
-                                    en.e = hee[kq];
-                                    blist[at] = en;
-                                }
-                            }
-                        }
-                        if (take) {
-                            unsigned char *bp = pcodes + min(pos, 35);
-                            *bp = static_cast<unsigned char>(*bp - sgn_c);
-                            if (pkerr) pkerr[kq] = __fmul_rn(__int2float_rn(hee[kq] - sgn_c * kOne), 0x1p-30f);
-                        }
-                    }
+                // The thread only says that it is concerned: the channel warp, which has the time, looks up the
+                // details and does the flips when it completes the channel.  (A queue that is full - a channel
+                // with hundreds of flips - leaves the thread to do its own.)
+                const int at = atomicAdd(&ctrl->qcount[pb], 1);
+                if (at < kStreamQueueCap) {
+                    ctrl->queue[pb][at] = static_cast<unsigned short>(qt);
+                } else {
+                    stream_flip_thread(qt, D, ctrl->T[pb], hs + pj * kStreamHeldBytes,
+                                       smem + lay.off_codes + static_cast<size_t>(pj) * lay.c_bytes, ctrl->kprev[pj],
+                                       reinterpret_cast<StreamListEntry *>(smem + lay.off_list) + pb * kStreamListCap, &ctrl->lcount[pb]);
                 }
             }
         };
@@ -495,13 +519,6 @@ squant_stream_kernel(const __grid_constant__ LaunchTable tbl, int qmax, unsigned
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&ctrl->qdone[b]);
                 break;
-            }
-            // A thread whose previous kernels have a strong candidate will probably be asked for their details at
-            // the end of this step: bring them from the scratch area (L2) into L1 meanwhile - no registers involved.
-            if (held.have && max(held.vmax, -held.vmin) >= kHalf) {
-                asm volatile("prefetch.global.L1 [%0];" ::"l"(held_v(b ^ 1)));
-                asm volatile("prefetch.global.L1 [%0];" ::"l"(held_e(b ^ 1)));
-                asm volatile("prefetch.global.L1 [%0];" ::"l"(held_i(b ^ 1)));
             }
             const bool active = qt < cur.quads;
             const unsigned char *wbuf = smem + static_cast<size_t>(b) * lay.w_bytes;
@@ -615,9 +632,9 @@ squant_stream_kernel(const __grid_constant__ LaunchTable tbl, int qmax, unsigned
             __syncwarp();
             if (lane == 0) mbar_arrive(&ctrl->qdone[b]);
             // what SQuant-C may need of these kernels one step from now (threads without kernels hold zeros)
-            *held_e(b) = make_int4(e4[0], e4[1], e4[2], e4[3]);
-            *held_v(b) = make_int4(v4[0], v4[1], v4[2], v4[3]);
-            *held_i(b) = i4;
+            *held_e(j) = make_int4(e4[0], e4[1], e4[2], e4[3]);
+            *held_v(j) = make_int4(v4[0], v4[1], v4[2], v4[3]);
+            *held_i(j) = i4;
             held.vmax = max(max(v4[0], v4[1]), max(v4[2], v4[3]));
             held.vmin = min(min(v4[0], v4[1]), min(v4[2], v4[3]));
             held.have = true;
@@ -746,6 +763,19 @@ squant_stream_kernel(const __grid_constant__ LaunchTable tbl, int qmax, unsigned
             const LayerDesc &L = tbl.layers[f_layer];
             unsigned char *codes = smem + lay.off_codes + static_cast<size_t>(pj) * lay.c_bytes;
             float *kerr = L.kerr ? L.kerr + static_cast<size_t>(f_m) * L.N : nullptr;
+            {   // the threads that said they are concerned: their flips, their members of the boundary bin
+                const int qn = min(ctrl->qcount[pb], kStreamQueueCap);
+                if (qn > 0) {
+                    const StreamDecision Dp = ctrl->dec[pb];
+                    const unsigned long long Tp = ctrl->T[pb];
+                    const unsigned char *hset = held_scratch + static_cast<size_t>(blockIdx.x) * (kStreamHeldSets * kStreamHeldBytes) + pj * kStreamHeldBytes;
+                    StreamListEntry *bl = reinterpret_cast<StreamListEntry *>(smem + lay.off_list) + pb * kStreamListCap;
+                    for (int x = lane; x < qn; x += 32)
+                        stream_flip_thread(ctrl->queue[pb][x], Dp, Tp, hset, codes, kerr, bl, &ctrl->lcount[pb]);
+                }
+                __syncwarp();
+                if (lane == 0) ctrl->qcount[pb] = 0;
+            }
             if (f_listing) {   // the first `f_rem` of the bin's members are flipped
                 const StreamListEntry *blist = reinterpret_cast<const StreamListEntry *>(smem + lay.off_list) + pb * kStreamListCap;
                 const int cnt = min(ctrl->lcount[pb], kStreamListCap);
