@@ -49,7 +49,7 @@ def algorithmic_bytes(shapes) -> float:
 
 def source_digest() -> str:
     h = hashlib.sha256()
-    for f in ("squant_device.cuh", "squant_pipe.cuh"):   # the device code; squant.cu is host code only
+    for f in ("squant_device.cuh", "squant_pipe.cuh", "squant_stream.cuh"):   # the device code; squant.cu is host code only
         with open(os.path.join(ROOT, "paper_2202_07471_b200", "csrc", f), "rb") as fh:
             h.update(fh.read())
     return h.hexdigest()[:16]

@@ -119,20 +119,26 @@ int squant_quantize_layer(const squant_layer *layer, const squant_options *opt, 
 /*
  * Algorithm 1 on every layer of a model in one pass (the paper sums per-layer times and notes
  * that layers could be quantized in parallel, Sec. 4.2): ONE grouped kernel launch for all
- * layers, plus one launch of a pipelined kernel for those layers whose 3x3 output channels are
- * longer than 8192 weights (cin a multiple of 4 and at most 2048, SQuant-K on, absmax scales).
+ * layers, plus one launch of a persistent kernel for those layers whose 3x3 output channels are
+ * longer than 8192 weights (cin a multiple of 4 and at most 2048, SQuant-K on, absmax scales): the
+ * streaming kernel when only int8 codes are wanted, the pipelined kernel for packed or
+ * dequantized outputs.
  *
  *   layers, n_layers  host array of descriptors holding DEVICE pointers; n_layers >= 0
  *   opt               bits / mode / flags shared by all layers; NULL means 4 bit, E|K|C, narrow
  *   cuda_stream       a cudaStream_t (NULL = default stream)
  *
  * The launch table (layer descriptors) travels by value in the kernel's parameter space: the call
- * allocates no device memory, uploads nothing and never synchronises; more than 96 layers are
- * issued as several launches.  Host-side launch tables of recent calls are cached.  Outputs are
- * valid when the stream reaches the end of the launches.  The pipelined kernel hands out its
- * channels through a counter in device memory that belongs to the cached launch tables of these
- * exact descriptors: two calls with the SAME descriptors must not overlap on the GPU (they would
- * race on the outputs anyway); calls with different descriptors may.  All arguments are validated
+ * uploads nothing and never synchronises; more than 96 layers are issued as several launches.
+ * Host-side launch tables of recent calls are cached.  The only device memory the call ever
+ * allocates is the streaming kernel's scratch area (72 KB per multiprocessor, about 11 MB on a
+ * B200): at the FIRST call with given descriptors that has such layers, by cudaMalloc, kept with
+ * the cached launch tables and freed with them (callers that cannot allocate: see
+ * squant_quantize_layer_noalloc).  Outputs are valid when the stream reaches the end of the
+ * launches.  The persistent kernels hand out their channels through a counter in device memory
+ * that, like the scratch area, belongs to the cached launch tables of these exact descriptors:
+ * two calls with the SAME descriptors must not overlap on the GPU (they would race on the
+ * outputs anyway); calls with different descriptors may.  All arguments are validated
  * on the host first; a failed call launches nothing and writes nothing.  Returns SQUANT_OK or a
  * negative SQUANT_ERR_* code.
  */

@@ -567,7 +567,6 @@ __device__ __forceinline__ KernelOut kernel9_exact(const float *wk, float y, flo
 // reported.  The four largest keys come from a 3x3 sorting tableau: sort each triple (rows), then
 // the columns; an entry in row i, column j has at least i * j - 1 entries above it, so the top
 // four of nine lie in row 1, column 1 and position (2, 2) (28 operations).
-template <bool kStraight = false>
 __device__ __forceinline__ bool kernel9_select(const float (&Psf)[9], float ef, unsigned char *cb,
                                                int &e_out, int &v_out, unsigned &idx_out)
 {
@@ -611,17 +610,7 @@ __device__ __forceinline__ bool kernel9_select(const float (&Psf)[9], float ef, 
         unsigned char *p2 = cb + (~m2 & 15);
         *p2 = static_cast<unsigned char>(*p2 - ((ok & (jx >= 3u)) ? sgn : 0));
     }
-    if (kStraight) {
-        // ranks 3 and 4 by predicated loads and stores: no branch, so that a caller's consecutive
-        // kernels stay one straight piece of code (the instructions are skipped, not jumped over)
-        const unsigned a3 = smem_addr(cb + (~m3 & 15)), a4 = smem_addr(cb + (~m4 & 15));
-        asm volatile("{\n\t.reg .pred p3, p4;\n\t.reg .b32 t3, t4;\n\t"
-                     "setp.ne.u32 p3, %2, 0;\n\tsetp.ne.u32 p4, %3, 0;\n\t"
-                     "@p3 ld.shared.u8 t3, [%0];\n\t@p3 sub.u32 t3, t3, %4;\n\t@p3 st.shared.u8 [%0], t3;\n\t"
-                     "@p4 ld.shared.u8 t4, [%1];\n\t@p4 sub.u32 t4, t4, %4;\n\t@p4 st.shared.u8 [%1], t4;\n\t}"
-                     :: "r"(a3), "r"(a4), "r"(static_cast<unsigned>(ok & (jx >= 5u))), "r"(static_cast<unsigned>(ok & (jx == 7u))), "r"(sgn)
-                     : "memory");
-    } else if (ok & (jx >= 5u)) {
+    if (ok & (jx >= 5u)) {
         unsigned char *p3 = cb + (~m3 & 15);
         *p3 = static_cast<unsigned char>(*p3 - sgn);
         if (jx == 7u) {

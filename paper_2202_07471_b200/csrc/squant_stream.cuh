@@ -213,7 +213,7 @@ __device__ __forceinline__ bool stream_kernel(const float2 (&P2)[18], float ef, 
         const int el = 9 * KQ + i;
         Pk[i] = (el & 1) ? P2[el >> 1].y : P2[el >> 1].x;
     }
-    return kernel9_select<false>(Pk, ef, cq + 9 * KQ, e_out, v_out, idx_out);
+    return kernel9_select(Pk, ef, cq + 9 * KQ, e_out, v_out, idx_out);
 }
 
 // The kernels stream_kernel<KQ> reported (about one in 10^5 on random weights): settled exactly,

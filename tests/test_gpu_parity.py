@@ -362,6 +362,31 @@ def test_host_entry_point_several_chunks_against_the_checker():
             assert int(b.codes.min()) >= -7 and not torch.isnan(b.scales).any()   # every channel was written
 
 
+@pytest.mark.parametrize("n", [2048, 1500, 1028])
+def test_streaming_kernel_hundreds_of_channel_flips(n):
+    """Long 3x3 channels whose kernel sums all lean the same way: SQuant-C flips hundreds of kernels per
+    channel, with candidates spread over many histogram bins - far more threads are concerned than the
+    streaming kernel's queue holds (the rest do their own flips), and the boundary bin is ranked from the
+    list.  Weights sit on the 4-bit grid of scale 1/8 except one element per kernel, which is off the grid
+    by 0.25 .. 0.49 of a step (downwards in the odd channels)."""
+    rng = np.random.default_rng(n)
+    m = 6
+    w = rng.integers(-6, 7, size=(m, n, 9)).astype(np.float32) * 0.125
+    off = rng.uniform(0.25, 0.49, size=(m, n)).astype(np.float32) * 0.125
+    sign = np.where(np.arange(m) % 2 == 0, 1.0, -1.0).astype(np.float32)[:, None]
+    pos = rng.integers(0, 9, size=(m, n))
+    off_grid = rng.integers(-5, 6, size=(m, n)).astype(np.float32) * 0.125 + sign * off
+    np.put_along_axis(w, pos[:, :, None], off_grid[:, :, None], axis=2)
+    w[:, 0, 0] = 0.875   # absmax: scale 1/8 at 4 bit
+    w = w.reshape(m, n, 3, 3)
+    (b,) = run_gpu([w], 4, EKC)
+    assert_layer_equal(b, w, 4, EKC, tag=f"n {n}")
+    r = oracle.quantize_layer(w, bits=4, mode=EKC)
+    flips = int(np.abs(np.rint((oracle.quantize_layer(w, bits=4, mode=EK).kernel_err.astype(np.float64).sum(axis=1)))).min())
+    assert flips > 200, flips   # the case really has hundreds of flips per channel
+    assert np.all(np.abs(r.channel_err) <= 0.5)
+
+
 @pytest.mark.parametrize("bits,flags", [(2, sq.FLAG_NARROW_RANGE), (6, sq.FLAG_NARROW_RANGE), (4, 0), (8, 0)])
 def test_pipelined_kernel_optional_outputs_and_ranges(bits, flags):
     """Long 3x3 channels (pipelined kernel) without the optional outputs, at 2 and 6 bit, and
