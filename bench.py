@@ -242,9 +242,9 @@ def _to_host(bufs):
     return [(b.codes.cpu().numpy(), b.scales.cpu().numpy(), b.kernel_err.cpu().numpy(), b.channel_err.cpu().numpy()) for b in bufs]
 
 
-def time_model(sq, torch, bufs, bits, mode, stream, flush, reps=15):
+def time_model(sq, torch, bufs, bits, mode, stream, flush, reps=15, flags=None):
     """One call over all layers: median milliseconds with L2 flushed before every call, and warm."""
-    call = sq.ModelCall(bufs, bits=bits, mode=mode)
+    call = sq.ModelCall(bufs, bits=bits, mode=mode) if flags is None else sq.ModelCall(bufs, bits=bits, mode=mode, flags=flags)
     for _ in range(3):
         call.run(stream)
     out = {}
@@ -369,7 +369,22 @@ def run_cuda(args):
         cfgs["large_layer_one_layer_E|C"] = {"layers": 1, "weights": one.numel(), "bits": BITS, "ms_cold": t["cold"], "ms_warm": t["warm"],
                                              "weights_per_s_cold": one.numel() / (t["cold"] * 1e-3), "channels": ch, "mismatches": bad[0],
                                              "note": "checker compared on the first 256 output channels"}
-        del eb, one, flush
+        # packed int4 codes on the same layer (4 + 0.5 + 4/9 B per weight): long channels with packed or
+        # dequantized outputs take the pipelined kernel
+        pk = [sq.alloc_outputs(one, pack_int4=True)]
+        pflags = sq.FLAG_NARROW_RANGE | sq.FLAG_PACK_INT4
+        t = time_model(sq, torch, pk, BITS, sq.MODE_EKC, stream, flush, reps=7, flags=pflags)
+        import oracle
+        rp = oracle.quantize_layer(host[0].numpy()[:256], bits=BITS, mode=sq.MODE_EKC, flags=pflags)
+        pbad = int((pk[0].codes[:256].cpu().numpy() != rp.codes).any(1).sum()
+                   + (pk[0].kernel_err[:256].cpu().numpy().view(np.uint32) != rp.kernel_err.view(np.uint32)).any(1).sum())
+        palg = one.numel() * (4 + 0.5 + 4 / 9) + one.shape[0] * 8
+        cfgs["large_layer_one_layer_packed_int4"] = {
+            "layers": 1, "weights": one.numel(), "bits": BITS, "ms_cold": t["cold"], "ms_warm": t["warm"],
+            "weights_per_s_cold": one.numel() / (t["cold"] * 1e-3), "gbs_cold": palg / (t["cold"] * 1e-3) / 1e9,
+            "frac_of_measured_cold": palg / (t["cold"] * 1e-3) / 1e9 / peak, "channels": 256, "mismatches": pbad,
+            "note": "checker compared on the first 256 output channels"}
+        del eb, pk, one, flush
         r50 = cfgs["resnet50"]
         extra = {"configs": cfgs,
                  "resnet50_model_latency_ms": {"median": r50["ms_cold"], "weights": r50["weights"], "layers": r50["layers"],
