@@ -113,7 +113,8 @@ def test_kernels_the_fast_selection_hands_back(bits):
 
 @pytest.mark.parametrize("bits,mode", [(4, EKC), (8, EKC), (3, EK)])
 def test_long_3x3_channels_pipelined_kernel(bits, mode):
-    """Layers of long 3x3 channels (more than 8192 weights each) take the pipelined kernel: several
+    """Layers of long 3x3 channels (more than 8192 weights each) take the streaming kernel (int8 codes only;
+    the pipelined kernel when packed or dequantized outputs are wanted, see the tests of those): several
     such layers of different widths in one launch (one, a few and many more channels than the GPU
     has multiprocessors), next to layers that stay with the grouped kernel, with special channels
     (zero, single non-zero, constant, scales far outside the reciprocal's range, ties)."""
@@ -133,7 +134,7 @@ def test_long_3x3_channels_pipelined_kernel(bits, mode):
 
 
 def test_random_mixed_launches():
-    """Seeded random models mixing long 3x3 layers (pipelined kernel), short 3x3, 1x1 and odd kernel
+    """Seeded random models mixing long 3x3 layers (streaming kernel), short 3x3, 1x1 and odd kernel
     shapes, random bit widths and modes, each launched twice into the same buffers."""
     rng = np.random.default_rng(12345)
     for trial in range(12):
@@ -247,7 +248,7 @@ def test_more_layers_than_one_launch_table_holds():
 
 
 def test_more_long_channel_layers_than_one_launch_table_holds():
-    """The same for the pipelined kernel: 101 layers of long 3x3 channels, two launches."""
+    """The same for the streaming kernel: 101 layers of long 3x3 channels, two launches."""
     shapes = [(1 + (i % 3), 912 + 4 * (i % 11), 3, 3) for i in range(101)]
     ws = [W.random_layer(s, seed=3000 + i) for i, s in enumerate(shapes)]
     n0 = sq.squant_launch_count()
@@ -341,7 +342,7 @@ def test_dequantized_output():
 
 def test_host_entry_point_several_chunks_against_the_checker():
     """squant_quantize_model_host takes the layers in chunks of about 64 MB of weights whose
-    uploads, launches and downloads overlap on three streams.  Four layers of 75 MB (pipelined
+    uploads, launches and downloads overlap on three streams.  Four layers of 75 MB (streaming
     kernel), a small one and a 1x1 one give five chunks; every output is compared with the checker
     on a sample of whole channels of every layer, called twice (cached staging and plans)."""
     shapes = [(512, 2048, 3, 3)] * 4 + [(40, 64, 3, 3), (300, 1000, 1, 1)]
@@ -389,7 +390,7 @@ def test_streaming_kernel_hundreds_of_channel_flips(n):
 
 @pytest.mark.parametrize("bits,flags", [(2, sq.FLAG_NARROW_RANGE), (6, sq.FLAG_NARROW_RANGE), (4, 0), (8, 0)])
 def test_pipelined_kernel_optional_outputs_and_ranges(bits, flags):
-    """Long 3x3 channels (pipelined kernel) without the optional outputs, at 2 and 6 bit, and
+    """Long 3x3 channels (streaming kernel) without the optional outputs, at 2 and 6 bit, and
     without the narrow-range flag; one table holds a layer with fewer channels than the GPU has
     multiprocessors and one with many more."""
     shapes = [(9, 1024, 3, 3), (700, 912, 3, 3), (33, 2048, 3, 3)]
@@ -412,7 +413,7 @@ def test_pipelined_kernel_optional_outputs_and_ranges(bits, flags):
 
 def test_overlapping_calls_with_different_descriptors():
     """Calls with different descriptors may overlap on the GPU: two models (both with layers for
-    the pipelined kernel, each with its own work counter) on two streams, several rounds."""
+    the streaming kernel, each with its own work counter and scratch area) on two streams, several rounds."""
     wa = [W.random_layer((200, 1024, 3, 3), seed=61), W.random_layer((50, 64, 3, 3), seed=62)]
     wb = [W.random_layer((300, 912, 3, 3), seed=63), W.random_layer((64, 300, 1, 1), seed=64)]
     ba = [sq.alloc_outputs(torch.from_numpy(w).cuda()) for w in wa]
@@ -450,7 +451,7 @@ def _clip_scales(w, bits, lo=1.5, hi=4.0, seed=0):
 def test_caller_supplied_scales(bits, flags):
     """Algorithm 1 with its scale as an input: the clip of Sec. 2.2 fires, clipped elements are
     never flipped outward and kernels / channels can run out of candidates.  All kernel sizes, long
-    3x3 channels included (they leave the pipelined kernel), modes E, E|K, E|K|C and E|C on 1x1."""
+    3x3 channels included (they leave the persistent kernels), modes E, E|K, E|K|C and E|C on 1x1."""
     shapes = [(12, 64, 3, 3), (9, 7, 3, 3), (10, 300, 1, 1), (6, 2049, 1, 1), (8, 5, 5, 5), (16, 1, 3, 3), (5, 3, 7, 7),
               (4, 1024, 3, 3), (3, 33, 2, 2)]
     ws = [W.random_layer(s, seed=300 + i) for i, s in enumerate(shapes)]
@@ -526,7 +527,7 @@ def test_failure_path_status_word_and_expiring_wait():
         sq.squant_device_status()
     assert ei.value.code == -10
     sq.squant_device_status()
-    w = W.random_layer((40, 1024, 3, 3), seed=12)      # pipelined kernel: its work counters were reset with the status
+    w = W.random_layer((40, 1024, 3, 3), seed=12)      # streaming kernel: its work counters were reset with the status
     (b,) = run_gpu([w], 4, EKC)
     assert_layer_equal(b, w, 4, EKC)
 
