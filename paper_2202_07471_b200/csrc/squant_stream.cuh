@@ -247,6 +247,7 @@ __device__ __forceinline__ void stream_flip_thread(int t, const StreamDecision &
                                                    const unsigned char *hset, unsigned char *codes, float *kerr_row,
                                                    StreamListEntry *blist, int *lcount)
 {
+    SQ_DBG(t >= 0 && t < kStreamQuantThreads, 21);   // a quantizer thread's index
     // (written by another thread of this CTA two hand-overs ago: read past the L1)
     const int4 he = __ldcg(reinterpret_cast<const int4 *>(hset) + t);
     const int4 hv = __ldcg(reinterpret_cast<const int4 *>(hset + 16 * kStreamQuantThreads) + t);
@@ -259,6 +260,7 @@ __device__ __forceinline__ void stream_flip_thread(int t, const StreamDecision &
         const int a = hvv[kq] * sgn_c;
         if (a >= t_min) {
             const int n = 4 * t + kq;
+            SQ_DBG(((hidx >> (8 * kq)) & 15u) < 9u, 22);   // the candidate is one of the kernel's nine elements
             const int pos = 36 * t + 9 * kq + min(static_cast<int>((hidx >> (8 * kq)) & 15u), 8);
             bool take;
             if (D.kind == 2) {
@@ -512,6 +514,7 @@ squant_stream_kernel(const __grid_constant__ LaunchTable tbl, int qmax, unsigned
             // the channel's scale (the scale warp has been over its weights during the previous step)
             stream_wait(ctrl, &ctrl->sready[b], static_cast<unsigned>(u) & 1u);
             const StreamSlot cur = ctrl->slot[b];
+            SQ_DBG(cur.item < n_items && cur.quads >= 0 && cur.quads <= kStreamQuantThreads && cur.layer >= 0 && cur.layer < tbl.n_layers, 24);
             if (cur.item < 0) {
                 // the last channel's flips, then the end mark for the channel warp
                 if (held.have) apply(b ^ 1, static_cast<unsigned>((i - 1) >> 1) & 1u, (i + 3) & 3);
@@ -787,6 +790,7 @@ squant_stream_kernel(const __grid_constant__ LaunchTable tbl, int qmax, unsigned
                         rank += (o.a > me.a || (o.a == me.a && o.n < me.n)) ? 1 : 0;
                     }
                     if (rank < f_rem) {
+                        SQ_DBG(me.pos >= 0 && me.pos < L.NK && me.n >= 0 && me.n < L.N, 23);   // a listed candidate of this channel
                         unsigned char *bp = codes + min(max(me.pos, 0), lay.c_bytes - 1);
                         *bp = static_cast<unsigned char>(*bp - f_sgn);
                         if (kerr) kerr[me.n] = __fmul_rn(__int2float_rn(me.e - f_sgn * kOne), 0x1p-30f);

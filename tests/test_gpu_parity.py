@@ -594,13 +594,15 @@ def test_channels_wider_than_one_thread_block():
 def test_checked_build_finds_no_violation_on_small_cases():
     """The checked build of the library (every shared-memory / table index verified, each 3x3
     channel's error sum taken a second time from its final codes by plain division) runs the
-    sweep of small shapes, the 3x3 cases the fast selection hands back, and a cluster case:
-    no check fails, and its results are the regular build's."""
+    sweep of small shapes, the 3x3 cases the fast selection hands back, long 3x3 channels through the
+    streaming kernel, and a cluster case: no check fails, and its results are the regular build's."""
     from paper_2202_07471_b200 import build as lib_build
     import os
     if not os.path.exists(lib_build.LIB_DEBUG):
         pytest.skip("libsquant_debug.so has not been built")
     ws = [adversarial_layer(s, seed=9 + i) for i, s in enumerate(SWEEP_SHAPES)] + [redo_layer(64, 4, seed=4), redo_layer(2048, 4)]
+    # long 3x3 channels (streaming kernel): special channels, heavy ties (digit-by-digit selection), a partial last warp
+    ws += [adversarial_layer((150, 1000, 3, 3), seed=77), coarse(W.random_layer((5, 2048, 3, 3), seed=78), steps=24, div=4)]
     ref = run_gpu(ws, 4, EKC)
     sq.use_library(lib_build.LIB_DEBUG)
     try:
