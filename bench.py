@@ -301,10 +301,10 @@ def run_cuda(args):
     torch.cuda.synchronize()
     sampler.start()
     # The timed steps last a few milliseconds: too short for the clock sampler (NVML, every 2 ms).  The same
-    # launches run untimed for 150 ms right before them, with the sampler on, so that the clocks and throttle
+    # launches run untimed for 60 ms right before them, with the sampler on, so that the clocks and throttle
     # reasons reported are those of this workload under load; sampling goes on through the timed steps.
     t_settle = time.perf_counter()
-    while time.perf_counter() - t_settle < 0.15:
+    while time.perf_counter() - t_settle < 0.06:
         for _ in range(8):
             call.run(stream)
         torch.cuda.synchronize()
@@ -319,7 +319,7 @@ def run_cuda(args):
     launches = sq.squant_launch_count() - launches0
     D.barrier()
     clocks = sampler.stop()
-    clocks["window"] = "150 ms of the same launches right before the timed steps, and the timed steps"
+    clocks["window"] = "60 ms of the same launches right before the timed steps, and the timed steps"
     total_ms = D.max_over_ranks(outer[0].elapsed_time(outer[1]))
     kernel_ms = D.max_over_ranks(sum(a.elapsed_time(b) for a, b in ev) / steps)
     value = n_weights * world * steps / (total_ms * 1e-3)
