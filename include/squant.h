@@ -133,8 +133,8 @@ int squant_quantize_layer(const squant_layer *layer, const squant_options *opt, 
  * Host-side launch tables of recent calls are cached.  The only device memory the call ever
  * allocates is the streaming kernel's scratch area (72 KB per multiprocessor, about 11 MB on a
  * B200): at the FIRST call with given descriptors that has such layers, by cudaMalloc, kept with
- * the cached launch tables and freed with them (callers that cannot allocate: see
- * squant_quantize_layer_noalloc).  Outputs are valid when the stream reaches the end of the
+ * the cached launch tables and freed with them (so that first call belongs outside any stream
+ * capture; callers that cannot allocate at all: see squant_quantize_layer_noalloc).  Outputs are valid when the stream reaches the end of the
  * launches.  The persistent kernels hand out their channels through a counter in device memory
  * that, like the scratch area, belongs to the cached launch tables of these exact descriptors:
  * two calls with the SAME descriptors must not overlap on the GPU (they would race on the
