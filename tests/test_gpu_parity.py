@@ -363,6 +363,29 @@ def test_host_entry_point_several_chunks_against_the_checker():
             assert int(b.codes.min()) >= -7 and not torch.isnan(b.scales).any()   # every channel was written
 
 
+def test_one_call_three_kernels():
+    """One call whose layers go to three kernels: long 3x3 channels with plain codes (streaming kernel), long 3x3
+    channels with a dequantized output (pipelined kernel), short layers (grouped kernel); three launches per
+    call, every output compared with the checker, repeated (cached plans, work counters, scratch area)."""
+    shapes = [(300, 1024, 3, 3), (200, 2048, 3, 3), (64, 64, 3, 3), (100, 512, 1, 1), (37, 1400, 3, 3)]
+    ws = [adversarial_layer(s, seed=31 + i) for i, s in enumerate(shapes)]
+    for bits in (4, 8):
+        bufs = [sq.alloc_outputs(torch.from_numpy(w).cuda(), dequant=(i in (1, 4)), dequant_bf16=(i == 4)) for i, w in enumerate(ws)]
+        count0 = sq.squant_launch_count()
+        for rep in range(3):
+            for b in bufs:
+                b.codes.fill_(-128)
+            sq.squant_quantize_model(bufs, bits=bits, mode=EKC)
+            sq.squant_device_status()
+            for shp, w, b in zip(shapes, ws, bufs):
+                assert_layer_equal(b, w, bits, EKC, tag=f"{shp} bits {bits} rep {rep}")
+                if b.dequant is not None:
+                    r = oracle.quantize_layer(w, bits=bits, mode=EKC)
+                    want = r.codes.astype(np.float32) * r.scales.reshape(-1, 1, 1, 1)
+                    assert np.array_equal(b.dequant.cpu().numpy().view(np.uint32), want.view(np.uint32)), f"{shp}: dequant"
+        assert sq.squant_launch_count() - count0 == 9
+
+
 @pytest.mark.parametrize("n", [2048, 1500, 1028])
 def test_streaming_kernel_hundreds_of_channel_flips(n):
     """Long 3x3 channels whose kernel sums all lean the same way: SQuant-C flips hundreds of kernels per
