@@ -435,8 +435,14 @@ int launch_plan(const ParamPlan &p, cudaStream_t stream)
         const int grid = std::min(p.pipe_items[c], std::max(g_sm_count_by_device[device], 1));
         if (p.pipe_stream[c]) {
             const int smem = sq::stream_layout(p.pipe_set_stride[c], p.pipe_nmax[c]).total;
-            if (!p.pipe_scratch[c])
-                SQ_CUDA(cudaMalloc(&p.pipe_scratch[c], static_cast<size_t>(std::max(g_sm_count_by_device[device], 1)) * sq::kStreamHeldSets * sq::kStreamHeldBytes));
+            if (!p.pipe_scratch[c]) {
+                const size_t bytes = static_cast<size_t>(std::max(g_sm_count_by_device[device], 1)) * sq::kStreamHeldSets * sq::kStreamHeldBytes;
+                if (cudaMalloc(&p.pipe_scratch[c], bytes) != cudaSuccess) {
+                    cudaGetLastError();   // the failed allocation is reported by the return code, not left pending
+                    p.pipe_scratch[c] = nullptr;
+                    return SQUANT_ERR_NOMEM;
+                }
+            }
             sq::squant_stream_kernel<<<grid, sq::kStreamThreads, smem, stream>>>(p.pipe_tables[c], p.qmax, p.mode, p.pipe_items[c],
                                                                              p.pipe_slot[c], p.pipe_set_stride[c], p.pipe_nmax[c],
                                                                              static_cast<unsigned char *>(p.pipe_scratch[c]));
